@@ -1,0 +1,207 @@
+"""Pins for the oracle's schedule and DiT layers: Gaussian-posterior algebra, library routines
+(CPU torch, fp64), brute force, structural identities and the sizes the paper quotes."""
+import numpy as np
+import pytest
+import torch
+import torch.nn.functional as F
+
+import synth
+from oracle import dit, schedule, drafter
+
+torch.set_default_dtype(torch.float64)
+
+
+# ----------------------------------------------------------------------------- schedule
+@pytest.mark.parametrize("kind,N", [("linear", 50), ("respaced", 250)])
+def test_posterior_variance_is_the_gaussian_posterior(kind, N):
+    # beta~ must be the variance of q(x_{t-1} | x_t, x_0): precision = alpha/beta + 1/(1 - abar_prev).
+    sc = schedule.make(kind, N)
+    abar_prev = np.concatenate([[1.0], sc.abar[:-1]])
+    with np.errstate(divide="ignore"):
+        prec = sc.alphas / sc.betas + 1.0 / (1.0 - abar_prev)
+    assert np.allclose(sc.sigma2, 1.0 / prec, rtol=1e-12, atol=0)
+    assert sc.sigma2[0] == 0.0 and np.all(sc.sigma2[1:] > 0)
+    assert np.all(sc.sigma2 <= sc.betas + 1e-18)
+
+
+@pytest.mark.parametrize("kind,N", [("linear", 50), ("respaced", 250)])
+def test_mean_is_the_posterior_mean_for_the_true_noise(kind, N):
+    # With x_t = sqrt(abar) x0 + sqrt(1-abar) eps, Eq. ddpm_update's mean equals the posterior mean
+    # mu~(x_t, x0) = sqrt(abar_prev) beta/(1-abar) x0 + sqrt(alpha)(1-abar_prev)/(1-abar) x_t.
+    sc = schedule.make(kind, N)
+    rng = np.random.default_rng(0)
+    x0, eps = rng.standard_normal(9), rng.standard_normal(9)
+    for s in (0, 1, N // 2, N - 1):
+        xt = np.sqrt(sc.abar[s]) * x0 + np.sqrt(1 - sc.abar[s]) * eps
+        abar_prev = 1.0 if s == 0 else sc.abar[s - 1]
+        mu = (np.sqrt(abar_prev) * sc.betas[s] / (1 - sc.abar[s]) * x0
+              + np.sqrt(sc.alphas[s]) * (1 - abar_prev) / (1 - sc.abar[s]) * xt)
+        assert np.allclose(sc.mean(xt, eps, s), mu, rtol=1e-11, atol=1e-12)
+    assert np.allclose(sc.mean(x0, 0 * x0, 3), x0 / np.sqrt(sc.alphas[3]))
+
+
+def test_respaced_keeps_abar_of_the_full_schedule():
+    b, idx = schedule.respaced_betas(250)
+    full = np.cumprod(1.0 - schedule.linear_betas(1000))
+    assert idx[0] == 0 and idx[-1] == 999 and np.all(np.diff(idx) >= 4) and np.all(np.diff(idx) <= 5)
+    assert np.allclose(np.cumprod(1.0 - b), full[idx], rtol=1e-12)
+    assert np.array_equal(schedule.make("respaced", 250).t_embed_value, idx)
+    lin = schedule.make("linear", 50)
+    assert lin.betas[0] == 1e-4 and np.isclose(lin.betas[-1], 2e-2) and lin.abar[-1] < 0.62
+
+
+# ----------------------------------------------------------------------------- layer primitives
+def test_primitives_against_torch():
+    rng = np.random.default_rng(1)
+    x = rng.standard_normal((7, 48)) * 3 + 0.5
+    t = torch.from_numpy(x)
+    assert np.allclose(dit.layer_norm(x), F.layer_norm(t, (48,), eps=1e-6).numpy(), atol=1e-12)
+    assert np.allclose(dit.gelu_tanh(x), F.gelu(t, approximate="tanh").numpy(), atol=1e-12)
+    assert np.allclose(dit.silu(x), F.silu(t).numpy(), atol=1e-12)
+    W, b = rng.standard_normal((5, 48)), rng.standard_normal(5)
+    assert np.allclose(dit.linear(x, W, b), F.linear(t, torch.from_numpy(W), torch.from_numpy(b)).numpy(), atol=1e-12)
+
+
+def test_attention_against_brute_force_and_torch():
+    rng = np.random.default_rng(2)
+    T, dh = 11, 6
+    q, k, v = (rng.standard_normal((T, dh)) for _ in range(3))
+    out = dit.attention(q, k, v)
+    brute = np.zeros((T, dh))
+    for i in range(T):
+        wts = np.array([np.exp(sum(q[i, c] * k[j, c] for c in range(dh)) / np.sqrt(dh)) for j in range(T)])
+        assert np.isclose((wts / wts.sum()).sum(), 1.0)
+        for j in range(T):
+            brute[i] += wts[j] / wts.sum() * v[j]
+    assert np.allclose(out, brute, atol=1e-12)
+    ref = F.scaled_dot_product_attention(*(torch.from_numpy(a)[None, None] for a in (q, k, v)))[0, 0].numpy()
+    assert np.allclose(out, ref, atol=1e-12)
+
+
+def test_multi_head_split_against_torch():
+    rng = np.random.default_rng(3)
+    T, D, h = 9, 24, 3
+    x = rng.standard_normal((T, D))
+    W, b = rng.standard_normal((3 * D, D)) * 0.2, rng.standard_normal(3 * D) * 0.1
+    out = dit.multi_head_attention(x, W, b, h)
+    qkv = F.linear(torch.from_numpy(x), torch.from_numpy(W), torch.from_numpy(b)).reshape(T, 3, h, D // h).permute(1, 2, 0, 3)
+    ref = F.scaled_dot_product_attention(qkv[0][None], qkv[1][None], qkv[2][None])[0].permute(1, 0, 2).reshape(T, D)
+    assert np.allclose(out, ref.numpy(), atol=1e-12)
+
+
+def test_patch_embed_is_a_strided_convolution_and_unpatchify_inverts_layout():
+    sh = synth.TINY
+    w = synth.make_target_weights(sh, 5)
+    x = synth.normal(5, 99, (sh.C, sh.H, sh.W)).astype(np.float64)
+    tok = dit.linear(dit.patchify(x, sh), w["pe_w"], w["pe_b"])
+    conv = F.conv2d(torch.from_numpy(x)[None], torch.from_numpy(w["pe_w"].astype(np.float64)).reshape(sh.D, sh.C, sh.patch, sh.patch),
+                    torch.from_numpy(w["pe_b"].astype(np.float64)), stride=sh.patch)[0]
+    assert np.allclose(tok, conv.flatten(1).T.numpy(), atol=1e-12)
+    # unpatchify: token (i,j), entry (p,q,c) lands at channel c, pixel (i*P+p, j*P+q)
+    g, P, co = sh.H // sh.patch, sh.patch, sh.c_out
+    t = np.arange(sh.n_tok * sh.out_dim, dtype=np.float64).reshape(sh.n_tok, sh.out_dim)
+    img = dit.unpatchify(t, sh)
+    for (i, j, p, q, c) in [(0, 0, 0, 0, 0), (1, 2, 1, 0, 3), (3, 3, 1, 1, 7), (2, 0, 0, 1, 5)]:
+        assert img[c, i * P + p, j * P + q] == t[i * g + j, (p * P + q) * co + c]
+
+
+def test_timestep_features_and_position_table():
+    f = dit.timestep_features(37.0, 256)
+    assert f.shape == (256,) and np.isclose(f[0], np.cos(37.0)) and np.isclose(f[128], np.sin(37.0))
+    assert np.isclose(f[127], np.cos(37.0 * 10000 ** (-127 / 128))) and np.allclose(f[:128] ** 2 + f[128:] ** 2, 1)
+    pos = synth.pos_embed_2d(synth.TINY)
+    assert pos.shape == (16, 64) and np.allclose(pos[0, :16], 0) and np.allclose(pos[0, 16:32], 1)
+    assert np.isclose(pos[5, 0], np.sin(1.0), atol=1e-6) and np.isclose(pos[5, 32], np.sin(1.0), atol=1e-6)  # token 5 = (row 1, col 1)
+    assert np.isclose(pos[6, 32], np.sin(2.0), atol=1e-6)
+
+
+# ----------------------------------------------------------------------------- structure
+def _tiny(seed=1, **kw):
+    sh = synth.TINY
+    return sh, synth.make_target_weights(sh, seed, **kw)
+
+
+def test_zero_gates_make_blocks_the_identity():
+    sh, w = _tiny()
+    D = sh.D
+    w = {k: v.copy() for k, v in w.items()}
+    for j in (2, 5):                       # gate rows of the modulation regressor
+        w["ada_w"][:, j * D:(j + 1) * D] = 0
+        w["ada_b"][:, j * D:(j + 1) * D] = 0
+    x = synth.normal(1, 50, (sh.C, sh.H, sh.W))
+    _, f = dit.forward(w, sh, x, 10.0, 3)
+    assert np.allclose(f, dit.embed(w, sh, x), atol=1e-14)
+
+
+def test_zero_head_gives_zero_noise_and_scaled_state():
+    sh, w = _tiny(out_gain=0.0)
+    sc = schedule.make("linear", 50)
+    x = synth.normal(1, 51, (1, sh.C, sh.H, sh.W))
+    means, eps, _ = dit.verify_pass(w, sh, sc, x, [7], [2], 0.0)
+    assert np.all(eps == 0) and np.allclose(means[0], x[0] / np.sqrt(sc.alphas[7]))
+
+
+def test_block_against_torch_functional_ops():
+    sh, w = _tiny(ada_std=0.3)
+    W = dit._with_heads(w, sh)
+    rng = np.random.default_rng(4)
+    x, sc = rng.standard_normal((sh.n_tok, sh.D)), rng.standard_normal(sh.D)
+    got = dit.block(x, sc, W, 1)
+    T = lambda a: torch.from_numpy(np.asarray(a, np.float64))
+    xt, D, h = T(x), sh.D, sh.heads
+    mod = F.linear(T(sc), T(w["ada_w"][1]), T(w["ada_b"][1])).chunk(6)
+    hh = F.layer_norm(xt, (D,), eps=1e-6) * (1 + mod[1]) + mod[0]
+    qkv = F.linear(hh, T(w["qkv_w"][1]), T(w["qkv_b"][1])).reshape(-1, 3, h, D // h).permute(1, 2, 0, 3)
+    a = F.scaled_dot_product_attention(qkv[0][None], qkv[1][None], qkv[2][None])[0].permute(1, 0, 2).reshape(-1, D)
+    xt = xt + mod[2] * F.linear(a, T(w["proj_w"][1]), T(w["proj_b"][1]))
+    hh = F.layer_norm(xt, (D,), eps=1e-6) * (1 + mod[4]) + mod[3]
+    hh = F.linear(F.gelu(F.linear(hh, T(w["fc1_w"][1]), T(w["fc1_b"][1])), approximate="tanh"), T(w["fc2_w"][1]), T(w["fc2_b"][1]))
+    xt = xt + mod[5] * hh
+    assert np.allclose(got, xt.numpy(), atol=1e-12)
+
+
+def test_guidance_combination():
+    sh, w = _tiny(ada_std=0.3, out_gain=5.0)
+    x = synth.normal(1, 52, (sh.C, sh.H, sh.W))
+    e_c, _ = dit.forward(w, sh, x, 20.0, 4)
+    e_u, _ = dit.forward(w, sh, x, 20.0, sh.n_classes)
+    assert np.abs(e_c - e_u).max() > 1e-6
+    assert np.array_equal(dit.guided_eps(w, sh, x, 20.0, 4, 1.0)[0], e_c)
+    e4, f = dit.guided_eps(w, sh, x, 20.0, 4, 4.0)
+    assert np.allclose(e4, e_u + 4.0 * (e_c - e_u), atol=1e-15) and f.shape == (2, sh.n_tok, sh.D)
+
+
+def test_packed_states_are_independent_sequences():
+    sh, w = _tiny(ada_std=0.3)
+    sc = schedule.make("linear", 50)
+    x, t, y = synth.pack_states(3, 1, 4, (sh.C, sh.H, sh.W), 50, sh.n_classes)
+    m_all, _, _ = dit.verify_pass(w, sh, sc, x[0], t[0], y[0], 0.0)
+    m_one, _, _ = dit.verify_pass(w, sh, sc, x[0, 2:3], t[0, 2:3], y[0, 2:3], 0.0)
+    assert np.array_equal(m_all[2], m_one[0]) and len(set(t[0].tolist())) == 4
+
+
+# ----------------------------------------------------------------------------- sizes the paper quotes
+def test_sizes_quoted_by_the_paper():
+    xl = synth.DIT_XL2_512
+    assert abs(xl.n_params() / 1e6 - 676) < 2.0                      # "676M parameters"
+    assert 28e6 < xl.drafter_params(1) < 33e6                        # "~32M trainable parameters"
+    assert xl.n_tok == 1024 and abs(xl.n_tok * xl.D * 4 / 1e6 - 4.7) < 0.05     # "[1024, 1152] ... ~4.7MB in FP32"
+    ratio = xl.flops_per_sequence(depth=1) / xl.flops_per_sequence()
+    assert np.isclose(ratio, 1 / 28)                                 # one block of 28: "~1/28"
+    assert abs(xl.flops_per_sequence() / 1e12 - 1.049) < 0.005
+
+
+def test_drafter_reuses_target_embedding_and_is_one_block():
+    sh, w = _tiny(ada_std=0.3)
+    wd = synth.make_drafter_weights(sh, 9, ada_std=0.3)
+    rng = np.random.default_rng(6)
+    x, f = rng.standard_normal((sh.C, sh.H, sh.W)), rng.standard_normal((sh.n_tok, sh.D))
+    eps, f_next = drafter.forward(w, wd, sh, x, f, 12.0, 1)
+    # written out: fuse -> one block -> head
+    g = np.concatenate([dit.embed(w, sh, x), f], axis=1) @ wd["fc_w"].astype(np.float64).T + wd["fc_b"]
+    sc = dit.silu(dit.conditioning(w, sh, 12.0, 1))
+    h = dit.block(g, sc, dit._with_heads(wd, sh), 0)
+    assert np.allclose(f_next, h, atol=1e-14) and eps.shape == (sh.C, sh.H, sh.W)
+    # the feature half of the fusion layer matters, and so does the latent half
+    assert np.abs(drafter.forward(w, wd, sh, x, 0 * f, 12.0, 1)[1] - f_next).max() > 1e-3
+    assert np.abs(drafter.forward(w, wd, sh, 0 * x, f, 12.0, 1)[1] - f_next).max() > 1e-3

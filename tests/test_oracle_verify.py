@@ -1,0 +1,177 @@
+"""Pins for the oracle's verifier: closed forms, the appendix's identities, Monte-Carlo laws."""
+import numpy as np
+import pytest
+from scipy import stats
+
+from oracle import verify as V
+
+RNG = np.random.default_rng(1234)
+
+
+def _case(d, s=0.3, sigma2=0.04):
+    m = RNG.standard_normal(d)
+    m_hat = m + s * RNG.standard_normal(d)
+    x_hat = m_hat + np.sqrt(sigma2) * RNG.standard_normal(d)
+    return m, m_hat, x_hat, sigma2
+
+
+@pytest.mark.parametrize("d", [1, 3, 64, 1000])
+def test_closed_form_equals_density_ratio(d):
+    # Eq. qp: the closed form must equal the difference of the two Gaussian log-densities.
+    m, m_hat, x_hat, s2 = _case(d)
+    a = V.log_ratio(x_hat, m, m_hat, s2)
+    b = V.log_ratio_definition(x_hat, m, m_hat, s2)
+    assert abs(a - b) <= 1e-9 * max(1.0, abs(b))
+
+
+def test_density_ratio_against_scipy():
+    m, m_hat, x_hat, s2 = _case(5)
+    ref = (stats.multivariate_normal(m, s2 * np.eye(5)).logpdf(x_hat)
+           - stats.multivariate_normal(m_hat, s2 * np.eye(5)).logpdf(x_hat))
+    assert abs(V.log_ratio(x_hat, m, m_hat, s2) - ref) < 1e-9 * max(1.0, abs(ref))
+
+
+def test_reflection_1d_mirrors_about_midpoint():
+    # Sec. 3.3: in one dimension x = 2 mid - x_hat.
+    m, m_hat, x_hat = np.array([0.3]), np.array([-1.1]), np.array([0.7])
+    assert np.allclose(V.reflect(x_hat, m, m_hat), m + m_hat - x_hat, atol=1e-15)
+
+
+def test_reflection_identities():
+    # Lemma 1 / Lemma 2: norm swaps, Re = -e, components orthogonal to e unchanged, involution.
+    m, m_hat, x_hat, _ = _case(37)
+    x = V.reflect(x_hat, m, m_hat)
+    assert np.isclose(np.linalg.norm(x - m), np.linalg.norm(x_hat - m_hat), rtol=1e-13)
+    assert np.isclose(np.linalg.norm(x - m_hat), np.linalg.norm(x_hat - m), rtol=1e-13)
+    e = (m_hat - m) / np.linalg.norm(m_hat - m)
+    r_in, r_out = x_hat - m_hat, x - m
+    assert np.isclose(e @ r_out, -(e @ r_in), rtol=1e-12)
+    assert np.allclose(r_out - e * (e @ r_out), r_in - e * (e @ r_in), atol=1e-13)
+    # reflecting back with the roles of the two means swapped returns the draft
+    assert np.allclose(V.reflect(x, m_hat, m), x_hat, atol=1e-12)
+    # the mirror image of x_hat across the hyperplane through mid with normal e
+    mid = 0.5 * (m + m_hat)
+    assert np.allclose(x, x_hat - 2 * e * (e @ (x_hat - mid)), atol=1e-12)
+
+
+def test_equal_means_always_accept_and_identity():
+    m, _, _, s2 = _case(16)
+    x_hat = m + 0.2 * RNG.standard_normal(16)
+    for u in (0.0, 1e-30, 0.5, 1.0 - 1e-16, 1.0):
+        x, ok, ell = V.verification(m, m, s2, x_hat, u)
+        assert ok and ell == 0.0 and np.array_equal(x, x_hat)
+    assert np.array_equal(V.reflect(x_hat, m, m), x_hat)
+
+
+@pytest.mark.parametrize("delta_over_sigma", [0.25, 1.0, 2.5])
+def test_acceptance_rate_matches_closed_form(delta_over_sigma):
+    # Appendix D: E[a] = 2 Phi(-||m_p - m_q|| / (2 sigma)); rejection rate = total variation (Theorem 1).
+    d, n, sigma = 6, 40000, 0.7
+    rng = np.random.default_rng(7)
+    m = rng.standard_normal(d)
+    direction = rng.standard_normal(d)
+    m_hat = m + delta_over_sigma * sigma * direction / np.linalg.norm(direction)
+    acc = 0
+    for _ in range(n):
+        x_hat = m_hat + sigma * rng.standard_normal(d)
+        acc += V.verification(m_hat, m, sigma ** 2, x_hat, rng.random())[1]
+    expect = 2.0 * stats.norm.cdf(-delta_over_sigma / 2.0)
+    se = np.sqrt(expect * (1 - expect) / n)
+    assert abs(acc / n - expect) < 4.5 * se
+
+
+def test_output_is_distributed_as_target():
+    # Unbiasedness (Appendix B): the output is N(m, sigma^2 I) although the draft is N(m_hat, .).
+    d, n, sigma = 4, 20000, 0.5
+    rng = np.random.default_rng(11)
+    m = rng.standard_normal(d)
+    m_hat = m + np.array([0.6, -0.3, 0.1, 0.4])
+    e = (m_hat - m) / np.linalg.norm(m_hat - m)
+    out = np.empty((n, d))
+    rejected = 0
+    for i in range(n):
+        x_hat = m_hat + sigma * rng.standard_normal(d)
+        out[i], ok, _ = V.verification(m_hat, m, sigma ** 2, x_hat, rng.random())
+        rejected += not ok
+    assert rejected > n // 10          # the test exercises the reflection branch
+    for c in range(d):
+        assert stats.kstest((out[:, c] - m[c]) / sigma, "norm").pvalue > 1e-3
+    assert stats.kstest(((out - m) @ e) / sigma, "norm").pvalue > 1e-3
+    # a verifier that skipped the reflection (kept the mean-shifted draft) must fail this pin
+    biased = m_hat + sigma * rng.standard_normal((n, d))
+    assert stats.kstest(((biased - m) @ e) / sigma, "norm").pvalue < 1e-6
+
+
+def test_relaxation_scale():
+    m, m_hat, x_hat, s2 = _case(50, s=0.2)
+    ell1 = V.log_ratio(x_hat, m, m_hat, s2, 1.0)
+    assert V.log_ratio(x_hat, m, m_hat, s2) == ell1                       # lambda = 1 is the strict rule
+    for lam in (0.5, 0.1, 0.0):
+        assert np.isclose(V.log_ratio(x_hat, m, m_hat, s2, lam), lam * ell1, rtol=1e-12, atol=1e-300)
+    # lambda -> 0 accepts everything; acceptance is monotone as lambda shrinks when ell < 0
+    if ell1 < 0:
+        u = np.exp(0.5 * ell1)        # rejected at lambda = 1
+        oks = [V.verification(m_hat, m, s2, x_hat, u, lam)[1] for lam in (1.0, 0.75, 0.5, 0.25, 0.0)]
+        assert oks[0] is False and oks[-1] is True
+        assert all(b >= a for a, b in zip(oks, oks[1:]))
+    # the reflection does not depend on lambda (e is a unit vector)
+    xr1 = V.verification(m_hat, m, s2, x_hat, 1.0, 1.0)[0]
+    xr2 = V.verification(m_hat, m, s2, x_hat, 1.0, 0.999)[0]
+    if ell1 < 0:
+        assert np.array_equal(xr1, xr2)
+
+
+def _brute_first_reject(m, m_hat, x_hat, s2, u, lam, n_valid):
+    B, K = u.shape
+    n_acc = np.zeros(B, dtype=np.int32)
+    for b in range(B):
+        flags = []
+        for k in range(n_valid[b]):
+            ratio = np.exp(min(0.0, lam[b, k] * V.log_ratio_definition(x_hat[b, k], m[b, k], m_hat[b, k], s2[b, k])))
+            flags.append(u[b, k] <= ratio)
+        n_acc[b] = flags.index(False) if False in flags else len(flags)
+    return n_acc
+
+
+def test_first_reject_scan_against_brute_force():
+    B, K, d = 40, 6, 24
+    rng = np.random.default_rng(3)
+    m = rng.standard_normal((B, K, d))
+    m_hat = m + 0.15 * rng.standard_normal((B, K, d))
+    s2 = rng.uniform(0.01, 0.1, (B, K))
+    x_hat = m_hat + np.sqrt(s2)[..., None] * rng.standard_normal((B, K, d))
+    u = rng.random((B, K))
+    lam = rng.uniform(0.2, 1.0, (B, K))
+    n_valid = rng.integers(0, K + 1, B)
+    x_out, n_acc, ell = V.spec_verify(m, m_hat, x_hat, s2, u, lam, n_valid)
+    assert np.array_equal(n_acc, _brute_first_reject(m, m_hat, x_hat, s2, u, lam, n_valid))
+    assert 0 < n_acc.sum() < n_valid.sum()
+    for b in range(B):
+        j = n_acc[b]
+        if n_valid[b] == 0:
+            assert np.all(x_out[b] == 0)
+        elif j == n_valid[b]:
+            assert np.array_equal(x_out[b], x_hat[b, j - 1])
+        else:
+            assert np.allclose(x_out[b], V.reflect(x_hat[b, j], m[b, j], m_hat[b, j]))
+            assert np.all(np.isnan(ell[b, j + 1:]))
+
+
+def test_first_reject_extreme_uniforms():
+    B, K, d = 5, 4, 8
+    rng = np.random.default_rng(5)
+    m = rng.standard_normal((B, K, d))
+    m_hat = m + rng.standard_normal((B, K, d))
+    s2 = np.full((B, K), 0.05)
+    x_hat = m_hat + np.sqrt(0.05) * rng.standard_normal((B, K, d))
+    _, n_acc, _ = V.spec_verify(m, m_hat, x_hat, s2, np.zeros((B, K)))
+    assert np.all(n_acc == K)                                   # u = 0 accepts everything
+    _, n_acc, ell = V.spec_verify(m, m_hat, x_hat, s2, np.ones((B, K)))
+    for b in range(B):                                          # u = 1 accepts iff ell >= 0
+        full = [V.log_ratio(x_hat[b, k], m[b, k], m_hat[b, k], 0.05) >= 0 for k in range(K)]
+        assert n_acc[b] == (full.index(False) if False in full else K)
+
+
+def test_sigma_must_be_positive():
+    with pytest.raises(ValueError):
+        V.verification(np.zeros(2), np.ones(2), 0.0, np.zeros(2), 0.5)
