@@ -1,0 +1,288 @@
+"""Benchmark of the packed parallel-verification path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload round|verifier] [--impl reference]
+
+One JSON line on stdout (rank 0).  A "step" is one pass of the hot path over one batch of synthetic
+input resident in HBM; `e2e` repeats it from pinned HOST buffers with the copies inside the timed
+region.  `--impl reference` times the CPU oracle on a bounded sample of the same workload.
+Multi-GPU runs shard whole batches across ranks (weak scaling, no data-path collective).
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--workload", default="default")
+    ap.add_argument("--batch", type=int, default=0, help="images per step (0 = workload default)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.FIELDS}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        rows = [r.strip().split(", ") for r in open(self.f.name) if r.strip()]
+        os.unlink(self.f.name)
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 8:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); power.append(float(r[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, r[4:8]):
+                if v.strip().lower().startswith("active"):
+                    reasons.add(nm)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": float(max(power))}
+
+
+# ------------------------------------------------------------------------------------------------
+# workloads: each provides device-resident steps, host-buffer steps, algorithmic work and an oracle sample
+# ------------------------------------------------------------------------------------------------
+class VerifierWorkload:
+    """Largest point of the standalone verifier sweep: d = 4x64x64, K = 16 drafts, B = 256 samples, fp32,
+    strict acceptance, target means N(0,1), draft = target + small offset, sigma2 from the 250-step schedule.
+    Inputs (805 MB) exceed L2, so consecutive steps cannot be served from cache."""
+    name = "verifier sweep point K=16 B=256 d=16384 strict"
+    metric, unit, dtype = "verifier HBM GB/s", "GB/s", "f32"
+
+    def __init__(self, batch, rank):
+        import torch
+        import synth
+        import paper_2511_20390_b200 as free
+        from paper_2511_20390_b200 import binding
+        self.torch, self.free, self.binding = torch, free, binding
+        self.B, self.K, self.d = (batch or 256), 16, 16384
+        sched = free.respaced_schedule(250)
+        s2 = np.tile(sched["sigma2"][np.linspace(240, 20, self.K).astype(int)].astype(np.float32), (self.B, 1))
+        m, mh, xh, u = synth.verifier_inputs(1000 + rank, self.B, self.K, self.d, 0.0015, s2)
+        self.host = dict(m=m, m_hat=mh, x_hat=xh, sigma2=s2, u=u)
+        self.dev = {k: torch.from_numpy(v).cuda() for k, v in self.host.items()}
+        self.x_out = torch.empty(self.B, self.d, device="cuda")
+        self.n_acc = torch.empty(self.B, dtype=torch.int32, device="cuda")
+        self.hv = None
+        # algorithmic bytes per sample: read m, m_hat, x_hat once, write one state, plus the [B,K] scalars
+        self.bytes_per_step = self.B * (3 * self.K * self.d * 4 + self.d * 4 + 12 * self.K)
+        self.units_per_step = self.bytes_per_step / 1e9          # GB
+        self.launches_per_step = 1
+        self.config = {"workload": self.name, "B": self.B, "K": self.K, "d": self.d,
+                       "cache": "inputs larger than L2 (805 MB per step)"}
+
+    def step(self):
+        d = self.dev
+        self.free.spec_verify(d["m"], d["m_hat"], d["x_hat"], d["sigma2"], d["u"], x_out=self.x_out, n_accept=self.n_acc)
+
+    def host_step(self):
+        if self.hv is None:
+            self.hv = self.binding.HostVerifier(self.B, self.K, self.d)
+            self.hv.load(**self.host)
+        self.hv.run()
+        return self.hv.h2d_bytes, self.hv.d2h_bytes
+
+    def roofline(self, ms_per_step, peaks):
+        ach = self.bytes_per_step / 1e9 / (ms_per_step / 1e3)
+        return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": ach / peaks["hbm_gbs"], "traffic": None, "kernel": "spec_verify_kernel",
+                "peak_source": peaks["source"]}
+
+    def oracle_sample(self):
+        from oracle import verify as ov
+        nb = 4
+        h = self.host
+        t0 = time.perf_counter()
+        ov.spec_verify(h["m"][:nb], h["m_hat"][:nb], h["x_hat"][:nb], h["sigma2"][:nb], h["u"][:nb])
+        dt = time.perf_counter() - t0
+        by = nb * (3 * self.K * self.d * 4 + self.d * 4 + 12 * self.K)
+        return by / 1e9 / dt, f"{nb} of {self.B} samples of the same batch, full K"
+
+
+def make_workload(name, batch, rank):
+    if name in ("verifier",):
+        return VerifierWorkload(batch, rank)
+    if name in ("default", "round"):
+        try:
+            from bench_round import RoundWorkload        # the full packed-verify round (DiT + verifier)
+        except ImportError:
+            return VerifierWorkload(batch, rank)
+        return RoundWorkload(batch, rank)
+    raise SystemExit(f"unknown workload {name}")
+
+
+def cpu_threads():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, rank):
+    """The CPU oracle, as it stands, on a bounded sample of the workload per step."""
+    if rank != 0:
+        return
+    os.environ.setdefault("CUDA_VISIBLE_DEVICES", "")
+    wl_name = args.workload
+    # the oracle needs no GPU: build host inputs only
+    import synth
+    from oracle import verify as ov
+    import importlib
+    cores = cpu_threads()
+    try:
+        br = importlib.import_module("bench_round")
+        out = br.reference_arm(args, cores)
+    except ImportError:
+        from paper_2511_20390_b200.schedule import respaced_schedule
+        B, K, d, nb = 256, 16, 16384, 2
+        s2 = np.tile(respaced_schedule(250)["sigma2"][np.linspace(240, 20, K).astype(int)].astype(np.float32), (nb, 1))
+        m, mh, xh, u = synth.verifier_inputs(1000, nb, K, d, 0.0015, s2)
+        by = nb * (3 * K * d * 4 + d * 4 + 12 * K)
+        for _ in range(args.warmup):
+            ov.spec_verify(m, mh, xh, s2, u)
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            ov.spec_verify(m, mh, xh, s2, u)
+        dt = (time.perf_counter() - t0) / args.steps
+        val = by / 1e9 / dt
+        out = {"metric": VerifierWorkload.metric, "value": val, "unit": "GB/s", "ms_per_step": dt * 1e3,
+               "dtype": "f64", "config": {"workload": VerifierWorkload.name},
+               "cpu_baseline": {"value": val, "unit": "GB/s", "cores": cores, "kind": "oracle",
+                                "sample": f"{nb} of {B} samples per step"}}
+    out.update({"impl": "reference", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "data": "synthetic",
+                "gpu_launches": 0})
+    out["e2e"] = {"value": out["value"], "unit": out["unit"], "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
+    print(json.dumps(out))
+
+
+def main():
+    args = parse()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        return run_reference(args, rank)
+
+    import torch
+    import torch.distributed as dist
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    import paper_2511_20390_b200 as free
+    free.lib()        # fail loudly if the CUDA library is not built
+
+    wl = make_workload(args.workload, args.batch, rank)
+    peaks = measured_peaks()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        wl.step()
+    barrier()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    stream = torch.cuda.current_stream()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for _ in range(args.steps):
+        wl.step()
+    ev1.record(stream)
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    kernel_ms = wl.kernel_ms_per_launch() if hasattr(wl, "kernel_ms_per_launch") else ms / args.steps
+    clocks = sampler.stop() if sampler else None
+
+    # end to end from pinned host buffers
+    for _ in range(2):
+        wl.host_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n_e2e = max(2, min(args.steps, 5))
+    e0.record(stream)
+    for _ in range(n_e2e):
+        h2d, d2h = wl.host_step()
+    e1.record(stream)
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+
+    if world > 1:
+        t = torch.tensor([ms, ms_e2e], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = t.tolist()
+    ms_step = ms / args.steps
+    value = wl.units_per_step * world / (ms_step / 1e3)
+    e2e_value = wl.units_per_step * world / (ms_e2e / n_e2e / 1e3)
+
+    if rank == 0:
+        out = {"metric": wl.metric, "value": value, "unit": wl.unit, "n_gpus": world, "steps": args.steps,
+               "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+               "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic", "config": wl.config,
+               "clocks": clocks,
+               "e2e": {"value": e2e_value, "unit": wl.unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+               "gpu_launches": wl.launches_per_step * args.steps,
+               "roofline": wl.roofline(kernel_ms, peaks)}
+        if hasattr(wl, "extra"):
+            out.update(wl.extra(ms_step, peaks))
+        if world == 1 and not args.no_cpu_baseline:
+            v, sample = wl.oracle_sample()
+            out["cpu_baseline"] = {"value": v, "unit": wl.unit, "cores": cpu_threads(), "kind": "oracle", "sample": sample}
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,246 @@
+/*
+ * free_b200 -- C ABI of the packed parallel-verification path of FREE
+ * ("Uncertainty-Aware Autoregression for Parallel Diffusion Transformers") for one B200 GPU.
+ *
+ * Conventions shared by every call
+ *   - Return value: 0 (FREE_OK) or a negative FREE_ERR_* code; free_strerror() names it.
+ *     No call throws, aborts or prints.
+ *   - Pointers marked DEVICE are addresses in the current CUDA device's global memory and must be
+ *     16-byte aligned; pointers marked HOST are ordinary host memory.  The caller owns every buffer.
+ *     The library allocates no device memory: scratch space is the caller's workspace `ws`, sized by
+ *     free_workspace_bytes().  Tensors are dense, row-major, innermost index last.
+ *   - `stream` is a cudaStream_t passed as void*.  Work is enqueued on it and the call returns
+ *     without waiting, except sample_trajectory(), which synchronises once per round.
+ *   - No random numbers are drawn inside: noise and uniforms are inputs, so that a run can be
+ *     reproduced by another implementation.
+ *   - "sequence" = one DiT forward of one latent state; with classifier-free guidance every state
+ *     costs G = 2 sequences (conditional, then unconditional with the null label), else G = 1.
+ *   - dtype FREE_FP32: all arithmetic in fp32 on CUDA cores (small models, exactness checks).
+ *     dtype FREE_BF16: GEMMs and attention on the tensor cores (tcgen05, bf16 operands, fp32
+ *     accumulation); residual stream, LayerNorm statistics, modulation and softmax in fp32.
+ */
+#ifndef FREE_B200_H
+#define FREE_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FREE_OK                   0
+#define FREE_ERR_ARG            (-1)   /* null pointer, negative count, bad enum                     */
+#define FREE_ERR_SHAPE          (-2)   /* dimensions inconsistent with the model or with each other  */
+#define FREE_ERR_ALIGN          (-3)   /* a DEVICE pointer is not 16-byte aligned                    */
+#define FREE_ERR_UNSUPPORTED    (-4)   /* valid request outside what the kernels implement           */
+#define FREE_ERR_SIGMA          (-5)   /* a variance was <= 0 or not finite                          */
+#define FREE_ERR_WORKSPACE      (-6)   /* workspace missing or smaller than free_workspace_bytes()   */
+#define FREE_ERR_CUDA           (-7)   /* a CUDA runtime / driver call failed                        */
+#define FREE_ERR_DEVICE_TIMEOUT (-8)   /* a bounded device-side wait gave up (pipeline fault)        */
+
+#define FREE_FP32 0
+#define FREE_BF16 1
+
+#define FREE_MAX_K 64                  /* most drafts per sample the verifier accepts */
+
+const char* free_strerror(int code);
+
+/* Weights of `n` stacked transformer blocks.  Matrices are [n, out, in] in the model's dtype
+ * (fp32 or bf16), biases are fp32 [n, out].  adaLN rows are ordered
+ * (shift1, scale1, gate1, shift2, scale2, gate2), each D wide.  All DEVICE. */
+typedef struct free_block_weights {
+    const void*  ada_w;  const float* ada_b;    /* [n, 6D, D], [n, 6D] */
+    const void*  qkv_w;  const float* qkv_b;    /* [n, 3D, D], [n, 3D]; output split as (3, heads, d_head) */
+    const void*  proj_w; const float* proj_b;   /* [n, D, D],  [n, D]  */
+    const void*  fc1_w;  const float* fc1_b;    /* [n, rD, D], [n, rD], r = mlp_ratio */
+    const void*  fc2_w;  const float* fc2_b;    /* [n, D, rD], [n, D]  */
+} free_block_weights;
+
+/* Target DiT (the paper uses DiT-XL/2 as published, Sec. 3.1 / Sec. 4; adaLN-Zero blocks). */
+typedef struct free_model_desc {
+    int32_t dtype;                       /* FREE_FP32 or FREE_BF16: type of the `void*` matrices and of features */
+    int32_t C, H, W, patch;              /* latent channels, height, width; patch size */
+    int32_t D, depth, heads;             /* hidden width, blocks, attention heads (D % heads == 0) */
+    int32_t n_classes;                   /* label n_classes is the null class */
+    int32_t c_out;                       /* output channels of the head (2C with learned variance; first C = noise) */
+    int32_t freq_dim, mlp_ratio;         /* sinusoidal timestep features (even), MLP expansion */
+    const void*  t_w1;  const float* t_b1;   /* [D, freq_dim], [D]   timestep MLP, layer 1 (then SiLU) */
+    const void*  t_w2;  const float* t_b2;   /* [D, D], [D]          timestep MLP, layer 2 */
+    const float* y_emb;                      /* [n_classes+1, D]     class embedding table */
+    const float* pe_w;  const float* pe_b;   /* [D, C*p*p], [D]      patch embedding, patch vector order (c, row, col) */
+    const float* pos;                        /* [n_tok, D]           fixed position table */
+    free_block_weights blocks;               /* n = depth */
+    const void*  fada_w; const float* fada_b;/* [2D, D], [2D]        final modulation (shift, scale) */
+    const float* fin_w;  const float* fin_b; /* [p*p*c_out, D], [..] head; output vector order (row, col, channel) */
+} free_model_desc;
+
+/* Drafter (Sec. 3.1): reuses the target's embedding tables; g = W_fc [embed(x) || f] + b_fc, then
+ * n_blocks DiT blocks (the paper uses one) and its own modulated head. */
+typedef struct free_drafter_desc {
+    int32_t n_blocks;
+    const void*  fc_w;   const float* fc_b;  /* [D, 2D], [D] */
+    free_block_weights blocks;
+    const void*  fada_w; const float* fada_b;
+    const float* fin_w;  const float* fin_b;
+} free_drafter_desc;
+
+/* Reverse-process tables indexed by schedule index s = 0..N-1 (s = N-1 is the noisiest), all DEVICE
+ * fp32 [N].  mean = coef_x[s] * x - coef_eps[s] * eps (Eq. ddpm_update, Appendix C);
+ * sigma2[s] is the fixed posterior variance (Sec. 4); t_embed_value[s] is fed to the timestep embedder. */
+typedef struct free_schedule {
+    int32_t N;
+    const float* coef_x;
+    const float* coef_eps;
+    const float* sigma2;
+    const float* t_embed_value;
+} free_schedule;
+
+typedef struct free_ctx free_ctx;
+
+/* Validate the descriptors, record them (weights are NOT copied: they must outlive the context) and
+ * prepare the tensor maps of the weight matrices.  `drafter` may be NULL.  HOST structs. */
+int free_create(const free_model_desc* target, const free_drafter_desc* drafter, free_ctx** out);
+int free_destroy(free_ctx* ctx);
+
+/* Bytes of workspace needed by dit_verify_pass / draft_step / sample_trajectory when at
+ * most `max_states` latent states are processed per call with guidance on (the larger case). */
+size_t free_workspace_bytes(const free_ctx* ctx, int max_states);
+
+/*
+ * dit_verify_pass -- the packed parallel target pass (Alg. 1, "compute means m_{a+1:b+1} in parallel";
+ * Sec. 3.3; Fig. 1a): ONE batched forward over n_states latent states, each with its own schedule
+ * index and label, followed by guidance and the reverse-transition mean (Eq. ddpm_update).
+ *   x_in      DEVICE fp32 [n_states, C, H, W]
+ *   t_idx     DEVICE int32 [n_states], schedule index of the transition each state undergoes
+ *   labels    DEVICE int32 [n_states] in 0..n_classes
+ *   cfg_scale guidance scale w: eps = eps_u + w (eps_c - eps_u); w <= 0 or w == 1 disables guidance (G = 1)
+ *   mean_out  DEVICE fp32 [n_states, C, H, W]          (required)
+ *   eps_out   DEVICE fp32 [n_states, C, H, W] or NULL  guided noise prediction
+ *   feat_out  DEVICE model dtype [n_states, G, n_tok, D] or NULL: top-block feature (token matrix after
+ *             the last block, Sec. 3.1), conditional stream first
+ * Errors: ARG, SHAPE (n_states < 1), ALIGN, WORKSPACE, UNSUPPORTED (model dims the kernels cannot tile), CUDA.
+ */
+int dit_verify_pass(free_ctx* ctx, int n_states,
+                         const float* x_in, const int32_t* t_idx, const int32_t* labels, float cfg_scale,
+                         const free_schedule* sched,
+                         float* mean_out, float* eps_out, void* feat_out,
+                         void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * spec_verify -- Algorithm 2 (reflection maximal coupling) applied to K drafts per sample in order,
+ * stopping at the first rejection (Alg. 1, verification loop), with the relaxed acceptance of
+ * Eq. acc_relax as a mode.  For draft k of sample b, with d = m_hat - m and r = x_hat - m_hat:
+ *     ell = -lambda (d.r + |d|^2 / 2) / sigma2      (= lambda (m - m_hat).(x_hat - mid) / sigma2, Eq. qp)
+ *     accept iff log u <= min(0, ell)               (u <= min(1, e^ell); u = 0 always accepts)
+ * At the first rejected draft j: x_out = m_j + r_j - 2 d_j (d_j.r_j) / |d_j|^2 (x_out = x_hat_j if d_j = 0).
+ * If all n_valid drafts are accepted x_out = x_hat of the last one.  Sums are accumulated in fp64.
+ *   B, K, d   samples, drafts per sample (1..FREE_MAX_K), elements per state
+ *   m_target, m_draft, x_draft  DEVICE fp32 [B, K, d]
+ *   sigma2    DEVICE fp32 [B, K]  variance of each transition (> 0)
+ *   lambda    DEVICE fp32 [B, K] relaxation scale in [0, 1], or NULL for the strict rule (lambda = 1)
+ *   u         DEVICE fp32 [B, K] uniforms in [0, 1]
+ *   n_valid   DEVICE int32 [B] number of drafts present (0..K), or NULL for K
+ *   x_out     DEVICE fp32 [B, d]; row b is left untouched when n_valid[b] == 0 or on a variance error
+ *   n_accept  DEVICE int32 [B]: number of accepted drafts (0..n_valid[b]); if < n_valid[b], draft
+ *             n_accept[b] (0-based) was the rejected one.  Set to FREE_ERR_SIGMA if a present draft
+ *             of that sample has sigma2 <= 0 or NaN.
+ *   logratio_out DEVICE fp32 [B, K] or NULL: ell of every present draft (NaN for absent ones)
+ * No workspace.  Errors: ARG, SHAPE (K out of range, d < 1), ALIGN, CUDA.
+ */
+int spec_verify(int B, int K, int64_t d,
+                     const float* m_target, const float* m_draft, const float* x_draft,
+                     const float* sigma2, const float* lambda, const float* u, const int32_t* n_valid,
+                     float* x_out, int32_t* n_accept, float* logratio_out, void* stream);
+
+/*
+ * draft_step -- one step of feature-level autoregression (Sec. 3.1; Alg. 1, drafting loop) for
+ * n_states states:  (m_hat, f_next) = p(. | x_prev, f_prev);  x_hat = m_hat + sqrt(sigma2[t]) * noise.
+ *   x_prev  DEVICE fp32 [n_states, C, H, W]
+ *   f_prev  DEVICE model dtype [n_states, G, n_tok, D]
+ *   t_idx, labels, cfg_scale, sched: as for dit_verify_pass (t_idx = the transition being predicted)
+ *   noise   DEVICE fp32 [n_states, C, H, W] standard normal draws
+ *   m_hat, x_hat  DEVICE fp32 [n_states, C, H, W]
+ *   f_next  DEVICE model dtype [n_states, G, n_tok, D] (may not alias f_prev)
+ * Errors: as dit_verify_pass, plus ARG if the context has no drafter.
+ */
+int draft_step(free_ctx* ctx, int n_states,
+                    const float* x_prev, const void* f_prev,
+                    const int32_t* t_idx, const int32_t* labels, float cfg_scale,
+                    const free_schedule* sched, const float* noise,
+                    float* m_hat, float* x_hat, void* f_next,
+                    void* ws, size_t ws_bytes, void* stream);
+
+typedef struct free_spec_params {
+    int32_t K;                 /* drafts per round (0 = plain sequential sampler) */
+    float   cfg_scale;
+    const float* lambda;       /* DEVICE fp32 [N] relaxation table indexed by transition n-1 (n = 1 first), or NULL = strict */
+} free_spec_params;
+
+typedef struct free_traj_stats {     /* HOST, filled on return */
+    int64_t rounds;                  /* batch rounds executed */
+    int64_t target_calls;            /* target invocations summed over samples (single steps + packed passes) */
+    int64_t draft_calls;             /* drafter steps summed over samples */
+    int64_t accepted, rejected;      /* drafts accepted / rejected, summed over samples */
+    int64_t accept_hist[FREE_MAX_K + 1];   /* rounds that accepted exactly i drafts */
+    double  parallel_efficiency;     /* B * N / target_calls (Sec. 4, metric 1) */
+} free_traj_stats;
+
+/*
+ * sample_trajectory -- Algorithm 1 for B samples with per-sample cursors.  N = sched->N transitions;
+ * transition n = 1..N uses schedule index N - n.  Each round: target step on the current state, K
+ * drafter steps, one packed target pass over (state, first K-1 drafts), sequential verification;
+ * the cursor moves past the last finalised state.  The final transition (sigma = 0) is never drafted.
+ *   x0            DEVICE fp32 [B, C, H, W]   initial latents ~ N(0, I)
+ *   labels        DEVICE int32 [B]
+ *   noise_target  DEVICE fp32 [B, N, C*H*W]  noise of transition n when taken by the target
+ *   noise_draft   DEVICE fp32 [B, N, C*H*W]  noise of transition n when proposed by the drafter
+ *   uniforms      DEVICE fp32 [B, N]         acceptance uniform of transition n
+ *   x_final       DEVICE fp32 [B, C, H, W]
+ *   stats         HOST, may be NULL
+ * Blocks until done.  Errors: as above; SIGMA if a drafted transition has sigma2 <= 0.
+ */
+int sample_trajectory(free_ctx* ctx, int B,
+                           const float* x0, const int32_t* labels,
+                           const free_schedule* sched, const free_spec_params* params,
+                           const float* noise_target, const float* noise_draft, const float* uniforms,
+                           float* x_final, free_traj_stats* stats,
+                           void* ws, size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Building blocks, exported so that each kernel can be checked against the CPU oracle on its own.
+ * They are the same kernels the calls above launch.
+ * ------------------------------------------------------------------------------------------------ */
+
+#define FREE_EPI_BIAS            0   /* out = acc + bias                                   */
+#define FREE_EPI_BIAS_GELU       1   /* out = gelu_tanh(acc + bias)                        */
+#define FREE_EPI_BIAS_SILU       2   /* out = silu(acc + bias)                             */
+#define FREE_EPI_GATE_RESIDUAL   3   /* resid[row, n] += gate[row / rows_per_seq, n] * (acc + bias), fp32 in place */
+
+/* out[M, N] = epilogue(A[M, K] * W[N, K]^T + bias[N]).  A, W in `dtype`; bias fp32 or NULL.
+ * out_dtype FREE_FP32 or FREE_BF16 (ignored for GATE_RESIDUAL, whose output is the fp32 `resid`).
+ * gate: DEVICE fp32, element (seq, n) at gate[seq * gate_stride + n].
+ * BF16 path (tcgen05): K % 64 == 0, N % 16 == 0; FP32 path (CUDA cores): any sizes.
+ * `ws` (>= free_op_linear_workspace_bytes()) holds the device error word of the pipeline. */
+size_t free_op_linear_workspace_bytes(void);
+int free_op_linear(int dtype, int epilogue, int out_dtype, int M, int N, int K,
+                   const void* A, const void* W, const float* bias, void* out,
+                   float* resid, const float* gate, int64_t gate_stride, int rows_per_seq,
+                   void* ws, size_t ws_bytes, void* stream);
+
+/* LayerNorm (no affine, eps 1e-6, biased variance) of each row of x fp32 [M, D], then
+ * y = ln * (1 + scale[seq]) + shift[seq], seq = row / rows_per_seq; shift/scale element (seq, c) at
+ * ptr[seq * mod_stride + c].  y in `out_dtype` [M, D]. */
+int free_op_ln_modulate(int out_dtype, int M, int D, int rows_per_seq, const float* x,
+                        const float* shift, const float* scale, int64_t mod_stride, void* y, void* stream);
+
+/* Non-causal multi-head self-attention of n_seq sequences: qkv [n_seq, n_tok, 3, heads, d_head] in
+ * `dtype`, out [n_seq, n_tok, heads * d_head] in `dtype`; softmax(q k^T / sqrt(d_head)) v per head. */
+int free_op_attention(int dtype, int n_seq, int n_tok, int heads, int d_head,
+                      const void* qkv, void* out, void* ws, size_t ws_bytes, void* stream);
+size_t free_op_attention_workspace_bytes(int dtype, int n_seq, int n_tok, int heads, int d_head);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FREE_B200_H */

@@ -1,0 +1,45 @@
+// Shared host/device helpers of the free_b200 library.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+#include "../../include/free_b200.h"
+
+#define FREE_CUDA_TRY(expr)                                   \
+    do {                                                      \
+        cudaError_t _e = (expr);                              \
+        if (_e != cudaSuccess) { (void)cudaGetLastError(); return FREE_ERR_CUDA; } \
+    } while (0)
+
+#define FREE_TRY(expr)                                        \
+    do { int _r = (expr); if (_r != FREE_OK) return _r; } while (0)
+
+static inline bool free_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static inline int free_check_launch() {
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? FREE_OK : FREE_ERR_CUDA;
+}
+
+static inline size_t free_round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+__device__ __forceinline__ float free_gelu_tanh(float a) {
+    // 0.5 a (1 + tanh(sqrt(2/pi) (a + 0.044715 a^3)))
+    const float k0 = 0.7978845608028654f, k1 = 0.044715f;
+    float t = tanhf(k0 * (a + k1 * a * a * a));
+    return 0.5f * a * (1.0f + t);
+}
+
+__device__ __forceinline__ float free_silu(float a) { return a / (1.0f + expf(-a)); }
+
+__device__ __forceinline__ float free_warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ double free_warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
