@@ -184,3 +184,168 @@ def spec_verify_host(m, m_hat, x_hat, sigma2, u, lam=None):
     x, n = hv.run()
     torch.cuda.current_stream().synchronize()
     return x.numpy().reshape((B,) + tuple(m.shape[2:])).copy(), n.numpy().copy()
+
+
+# ------------------------------------------------------------------------------------------ model
+_ACT = {FREE_FP32: torch.float32, FREE_BF16: torch.bfloat16}
+_MATRICES = ("t_w1", "t_w2", "ada_w", "qkv_w", "proj_w", "fc1_w", "fc2_w", "fada_w", "fc_w")
+
+
+class DeviceSchedule:
+    """The four reverse-process tables (see paper_2511_20390_b200.schedule) as fp32 device arrays."""
+
+    def __init__(self, tables: dict, device="cuda"):
+        self.N = int(len(tables["sigma2"]))
+        self.t = {k: torch.tensor(np.asarray(v, dtype=np.float32), device=device) for k, v in tables.items()}
+        self.desc = ScheduleDesc(self.N, *(self.t[k].data_ptr() for k in ("coef_x", "coef_eps", "sigma2", "t_embed_value")))
+
+
+def _upload(weights: dict, dtype: int, device):
+    out = {}
+    for k, v in weights.items():
+        t = torch.from_numpy(np.ascontiguousarray(v, dtype=np.float32)).to(device)
+        out[k] = t.to(_ACT[dtype]).contiguous() if k in _MATRICES else t
+    return out
+
+
+def _block_desc(w):
+    return BlockWeights(*(w[k].data_ptr() for k in ("ada_w", "ada_b", "qkv_w", "qkv_b", "proj_w", "proj_b",
+                                                    "fc1_w", "fc1_b", "fc2_w", "fc2_b")))
+
+
+class Model:
+    """A target DiT (and optionally a drafter) resident on the GPU, bound to a library context.
+
+    `shape` carries the dimensions (fields C, H, W, patch, D, depth, heads, n_classes, c_out, freq_dim,
+    mlp_ratio); `weights` / `drafter_weights` are dicts of host arrays laid out as the public header
+    describes.  dtype "fp32" or "bf16" selects the compute mode.
+    """
+
+    def __init__(self, shape, weights: dict, drafter_weights: dict | None = None, dtype: str = "bf16",
+                 n_draft_blocks: int = 1, device="cuda"):
+        self.shape, self.dtype = shape, {"fp32": FREE_FP32, "bf16": FREE_BF16}[dtype]
+        self.act = _ACT[self.dtype]
+        self.device = torch.device(device)
+        self.w = _upload(weights, self.dtype, self.device)
+        w = self.w
+        md = ModelDesc(self.dtype, shape.C, shape.H, shape.W, shape.patch, shape.D, shape.depth, shape.heads,
+                       shape.n_classes, shape.c_out, shape.freq_dim, shape.mlp_ratio,
+                       *(w[k].data_ptr() for k in ("t_w1", "t_b1", "t_w2", "t_b2", "y_emb", "pe_w", "pe_b", "pos")),
+                       _block_desc(w), *(w[k].data_ptr() for k in ("fada_w", "fada_b", "fin_w", "fin_b")))
+        dd = None
+        self.wd = None
+        if drafter_weights is not None:
+            self.wd = _upload(drafter_weights, self.dtype, self.device)
+            wd = self.wd
+            dd = DrafterDesc(n_draft_blocks, wd["fc_w"].data_ptr(), wd["fc_b"].data_ptr(), _block_desc(wd),
+                             *(wd[k].data_ptr() for k in ("fada_w", "fada_b", "fin_w", "fin_b")))
+        self.ctx = C.c_void_p()
+        _check(lib().free_create(C.byref(md), C.byref(dd) if dd is not None else None, C.byref(self.ctx)), "free_create")
+        self._ws = None
+
+    def __del__(self):
+        try:
+            if getattr(self, "ctx", None):
+                lib().free_destroy(self.ctx)
+                self.ctx = None
+        except Exception:
+            pass
+
+    def workspace(self, n_states: int):
+        need = lib().free_workspace_bytes(self.ctx, int(n_states))
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = None
+            self._ws = torch.empty(need, dtype=torch.uint8, device=self.device)
+        return self._ws
+
+    @staticmethod
+    def guided(cfg_scale: float) -> int:
+        return 2 if (cfg_scale > 0 and cfg_scale != 1.0) else 1
+
+    def dit_verify_pass(self, x, t_idx, labels, cfg_scale, sched: DeviceSchedule, want_eps=False, want_feat=False,
+                        mean_out=None):
+        """One packed target pass.  x: CUDA fp32 [n, C, H, W]; t_idx, labels: int32 [n].
+        Returns mean [n,C,H,W] (+ eps, + feat [n,G,n_tok,D] when asked)."""
+        sh = self.shape
+        n = x.shape[0]
+        _dev(x, torch.float32); _dev(t_idx, torch.int32); _dev(labels, torch.int32)
+        mean = torch.empty_like(x) if mean_out is None else mean_out
+        eps = torch.empty_like(x) if want_eps else None
+        feat = (torch.empty((n, self.guided(cfg_scale), sh.n_tok, sh.D), dtype=self.act, device=x.device)
+                if want_feat else None)
+        ws = self.workspace(n)
+        _check(lib().dit_verify_pass(self.ctx, n, _ptr(x), _ptr(t_idx), _ptr(labels), float(cfg_scale),
+                                     C.byref(sched.desc), _ptr(mean), _ptr(eps), _ptr(feat),
+                                     _ptr(ws), ws.numel(), _stream()), "dit_verify_pass")
+        out = (mean,) + ((eps,) if want_eps else ()) + ((feat,) if want_feat else ())
+        return out if len(out) > 1 else mean
+
+    def draft_step(self, x_prev, f_prev, t_idx, labels, cfg_scale, sched: DeviceSchedule, noise):
+        """One drafter step.  Returns (m_hat, x_hat, f_next)."""
+        n = x_prev.shape[0]
+        _dev(x_prev, torch.float32); _dev(f_prev, self.act); _dev(noise, torch.float32)
+        m_hat, x_hat, f_next = torch.empty_like(x_prev), torch.empty_like(x_prev), torch.empty_like(f_prev)
+        ws = self.workspace(n)
+        _check(lib().draft_step(self.ctx, n, _ptr(x_prev), _ptr(f_prev), _ptr(_dev(t_idx, torch.int32)),
+                                _ptr(_dev(labels, torch.int32)), float(cfg_scale), C.byref(sched.desc), _ptr(noise),
+                                _ptr(m_hat), _ptr(x_hat), _ptr(f_next), _ptr(ws), ws.numel(), _stream()), "draft_step")
+        return m_hat, x_hat, f_next
+
+    def sample_trajectory(self, x0, labels, sched: DeviceSchedule, K, cfg_scale, noise_target, noise_draft=None,
+                          uniforms=None, lam=None):
+        """Algorithm 1 for a batch.  Returns (x_final, stats dict)."""
+        B = x0.shape[0]
+        _dev(x0, torch.float32); _dev(labels, torch.int32); _dev(noise_target, torch.float32)
+        prm = SpecParams(int(K), float(cfg_scale), None if lam is None else _dev(lam, torch.float32).data_ptr())
+        st = TrajStats()
+        x_final = torch.empty_like(x0)
+        ws = self.workspace(B * max(int(K), 1))
+        _check(lib().sample_trajectory(self.ctx, B, _ptr(x0), _ptr(labels), C.byref(sched.desc), C.byref(prm),
+                                       _ptr(noise_target), _ptr(noise_draft), _ptr(uniforms), _ptr(x_final),
+                                       C.byref(st), _ptr(ws), ws.numel(), _stream()), "sample_trajectory")
+        stats = {k: getattr(st, k) for k in ("rounds", "target_calls", "draft_calls", "accepted", "rejected",
+                                             "parallel_efficiency")}
+        stats["accept_hist"] = list(st.accept_hist)[:int(K) + 1]
+        return x_final, stats
+
+
+# ------------------------------------------------------------------------------------------ single ops
+def op_linear(A, W, bias=None, epilogue=EPI_BIAS, out_dtype=None, resid=None, gate=None, rows_per_seq=1):
+    """epilogue(A W^T + bias) with the library's linear-layer kernel (fp32: CUDA cores, bf16: tcgen05)."""
+    dtype = FREE_FP32 if A.dtype == torch.float32 else FREE_BF16
+    M, K = A.shape
+    N = W.shape[0]
+    od = dtype if out_dtype is None else out_dtype
+    out = None if epilogue == EPI_GATE_RESIDUAL else torch.empty((M, N), dtype=_ACT[od], device=A.device)
+    ws = torch.zeros(lib().free_op_linear_workspace_bytes(), dtype=torch.uint8, device=A.device)
+    _check(lib().free_op_linear(dtype, epilogue, od, M, N, K, _ptr(A), _ptr(W), _ptr(bias), _ptr(out), _ptr(resid),
+                                _ptr(gate), 0 if gate is None else gate.stride(0), rows_per_seq,
+                                _ptr(ws), ws.numel(), _stream()), "free_op_linear")
+    err = int(ws[:4].view(torch.int32).item())
+    if err:
+        raise FreeError(-8, f"free_op_linear (device error word {err:#x})")
+    return resid if epilogue == EPI_GATE_RESIDUAL else out
+
+
+def op_ln_modulate(x, shift, scale, rows_per_seq, out_dtype=FREE_FP32):
+    M, D = x.shape
+    y = torch.empty((M, D), dtype=_ACT[out_dtype], device=x.device)
+    _check(lib().free_op_ln_modulate(out_dtype, M, D, rows_per_seq, _ptr(x), _ptr(shift), _ptr(scale),
+                                     shift.stride(0), _ptr(y), _stream()), "free_op_ln_modulate")
+    return y
+
+
+def op_attention(qkv, heads):
+    """qkv [n_seq, n_tok, 3*D] (split as 3, heads, d_head) -> [n_seq, n_tok, D]."""
+    dtype = FREE_FP32 if qkv.dtype == torch.float32 else FREE_BF16
+    n_seq, n_tok, D3 = qkv.shape
+    D = D3 // 3
+    out = torch.empty((n_seq, n_tok, D), dtype=qkv.dtype, device=qkv.device)
+    need = lib().free_op_attention_workspace_bytes(dtype, n_seq, n_tok, heads, D // heads)
+    ws = torch.zeros(need, dtype=torch.uint8, device=qkv.device)
+    _check(lib().free_op_attention(dtype, n_seq, n_tok, heads, D // heads, _ptr(qkv), _ptr(out), _ptr(ws), need, _stream()),
+           "free_op_attention")
+    err = int(ws[:4].view(torch.int32).item())
+    if err:
+        raise FreeError(-8, f"free_op_attention (device error word {err:#x})")
+    return out

@@ -1,0 +1,61 @@
+// Internal interfaces between the translation units of libfree_b200 (not part of the public ABI).
+#pragma once
+#include "common.cuh"
+
+// ---- linear layers ---------------------------------------------------------------------------
+// out = epilogue(A[M,K] * W[N,K]^T + bias).  A has row stride lda, W row stride ldw (elements).
+enum {
+    EPI_BIAS = FREE_EPI_BIAS,
+    EPI_BIAS_GELU = FREE_EPI_BIAS_GELU,
+    EPI_BIAS_SILU = FREE_EPI_BIAS_SILU,
+    EPI_GATE_RESIDUAL = FREE_EPI_GATE_RESIDUAL,   // resid += gate * (acc + bias); gate == nullptr means 1
+    EPI_BIAS_EMB_SILU = 4,                        // out = silu(acc + bias + emb[emb_idx[row], n])
+    EPI_QKV_HEADS = 5,                            // bf16 only: scatter (acc + bias) into head-major q, k and v^T
+};
+
+struct LinearArgs {
+    int M = 0, N = 0, K = 0;
+    const void* A = nullptr; long long lda = 0;
+    const void* W = nullptr; long long ldw = 0;
+    const float* bias = nullptr;
+    int epi = EPI_BIAS;
+    int out_dtype = FREE_FP32;
+    void* out = nullptr; long long ldo = 0;
+    float* resid = nullptr;                       // [M, N] fp32, row stride N
+    const float* gate = nullptr; long long gate_stride = 0; int rows_per_seq = 1;
+    const float* emb = nullptr; const int32_t* emb_idx = nullptr;
+    // EPI_QKV_HEADS
+    int heads = 0, d_head = 0, d_pad = 0, n_tok = 0;
+    void* q = nullptr; void* k = nullptr; void* vt = nullptr;
+    uint32_t* err = nullptr;                      // device error word (tensor-core path)
+};
+
+int linear_fp32(const LinearArgs& a, cudaStream_t s);   // CUDA cores, any sizes
+int linear_bf16(const LinearArgs& a, cudaStream_t s);   // tcgen05; K % 64 == 0, N % 16 == 0
+bool linear_bf16_supported(int N, int K);
+
+// ---- attention -------------------------------------------------------------------------------
+// token-major qkv [n_seq, n_tok, 3, heads, d_head] -> out [n_seq, n_tok, heads*d_head]
+int attention_simt(int dtype, int n_seq, int n_tok, int heads, int d_head, const void* qkv, void* out, cudaStream_t s);
+// head-major bf16 operands written by EPI_QKV_HEADS: q,k [n_seq, heads, n_tok, d_pad], vt [n_seq, heads, d_pad, n_tok]
+int attention_tc(int n_seq, int n_tok, int heads, int d_head, int d_pad, const void* q, const void* k, const void* vt,
+                 void* out, uint32_t* err, cudaStream_t s);
+bool attention_tc_supported(int n_tok, int d_head);
+int attention_tc_dpad(int d_head);
+
+// ---- elementwise / row kernels ----------------------------------------------------------------
+int cond_setup(int dtype, int n_states, int G, int freq_dim, int n_classes, int N_sched,
+               const int32_t* t_idx, const int32_t* labels, const float* t_embed_value,
+               void* temb /*[S,freq_dim]*/, int32_t* lab_seq /*[S]*/, cudaStream_t s);
+int patch_embed(int out_dtype, int n_states, int G, int C, int H, int W, int p, int D,
+                const float* x_in, long long x_stride, const float* pe_w, const float* pe_b, const float* pos,
+                void* out /*[S*n_tok, D]*/, cudaStream_t s);
+int ln_modulate(int out_dtype, int M, int D, int rows_per_seq, const float* x, const float* shift, const float* scale,
+                long long mod_stride, void* y, cudaStream_t s);
+int convert_rows(int out_dtype, long long n, const float* x, void* y, cudaStream_t s);
+int head_to_mean(int n_states, int G, int C, int H, int W, int p, int c_out, float cfg_scale, int N_sched,
+                 const float* head_out /*[S*n_tok, p*p*c_out]*/, const float* x_in, long long x_stride,
+                 const int32_t* t_idx, const float* coef_x, const float* coef_eps, const float* sigma2,
+                 float* mean_out, long long mean_stride, float* eps_out, long long eps_stride,
+                 const float* noise, long long noise_stride, float* sample_out, long long sample_stride,
+                 float* sample_out2, long long sample2_stride, const int32_t* sample2_mask, cudaStream_t s);

@@ -1,0 +1,248 @@
+// Bandwidth-bound row and elementwise kernels of the DiT pass: conditioning features, patch embedding,
+// LayerNorm + adaLN modulation, feature conversion, and the tail that turns the head's output into the
+// guided noise prediction and the reverse-transition mean (Eq. ddpm_update).
+#include "internal.h"
+#include <math.h>
+
+namespace {
+
+template <typename T> __device__ __forceinline__ void store_act(T* p, float v);
+template <> __device__ __forceinline__ void store_act<float>(float* p, float v) { *p = v; }
+template <> __device__ __forceinline__ void store_act<__nv_bfloat16>(__nv_bfloat16* p, float v) { *p = __float2bfloat16(v); }
+
+// ---------------------------------------------------------------------------------------------
+// Sinusoidal timestep features [cos(tau w_i), sin(tau w_i)], w_i = 10000^(-i/half), and the label of
+// every sequence (the unconditional stream of a guided state uses the null class).
+template <typename T>
+__global__ void cond_setup_kernel(int n_states, int G, int freq_dim, int n_classes, int N_sched,
+                                  const int32_t* t_idx, const int32_t* labels, const float* t_embed_value,
+                                  T* temb, int32_t* lab_seq) {
+    const int q = blockIdx.x;                 // sequence
+    const int st = q / G, g = q % G;
+    int t = t_idx[st];
+    t = t < 0 ? 0 : (t >= N_sched ? N_sched - 1 : t);
+    const double tau = (double)t_embed_value[t];
+    const int half = freq_dim / 2;
+    for (int i = threadIdx.x; i < half; i += blockDim.x) {
+        const double w = exp(-log(10000.0) * (double)i / (double)half);
+        store_act(temb + (size_t)q * freq_dim + i, (float)cos(tau * w));
+        store_act(temb + (size_t)q * freq_dim + half + i, (float)sin(tau * w));
+    }
+    if (threadIdx.x == 0) {
+        int y = labels[st];
+        y = y < 0 ? 0 : (y > n_classes ? n_classes : y);
+        lab_seq[q] = g == 0 ? y : n_classes;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Patch embedding: token (i, j) of a state gathers its C*p*p patch (order: channel, row, column),
+// out = pe_w . patch + pe_b + pos[token].  One CTA per (state, token); written once per guidance stream.
+template <typename T>
+__global__ void __launch_bounds__(128) patch_embed_kernel(int G, int C, int H, int W, int p, int D,
+                                                          const float* x_in, long long x_stride, const float* pe_w,
+                                                          const float* pe_b, const float* pos, T* out) {
+    extern __shared__ float patch[];
+    const int gw = W / p, n_tok = (H / p) * gw, pd = C * p * p;
+    const int st = blockIdx.x / n_tok, tok = blockIdx.x % n_tok;
+    const int ti = tok / gw, tj = tok % gw;
+    const float* x = x_in + (long long)st * x_stride;
+    for (int e = threadIdx.x; e < pd; e += blockDim.x) {
+        int c = e / (p * p), r = (e / p) % p, cc = e % p;
+        patch[e] = x[((long long)c * H + ti * p + r) * W + tj * p + cc];
+    }
+    __syncthreads();
+    for (int o = threadIdx.x; o < D; o += blockDim.x) {
+        const float* w = pe_w + (long long)o * pd;
+        float acc = 0.f;
+        for (int e = 0; e < pd; ++e) acc = fmaf(w[e], patch[e], acc);
+        acc += pe_b[o] + pos[(long long)tok * D + o];
+        for (int g = 0; g < G; ++g)
+            store_act(out + ((long long)(st * G + g) * n_tok + tok) * D + o, acc);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// LayerNorm (no affine, eps 1e-6, biased variance, two-pass statistics) + y = ln (1 + scale) + shift.
+// One warp per row.  VPL > 0: the row (D = 128 * VPL) lives in registers as VPL float4 per lane.
+template <typename T, int VPL>
+__global__ void __launch_bounds__(256) ln_modulate_kernel(int M, int D, int rows_per_seq, const float* x,
+                                                          const float* shift, const float* scale, long long mod_stride, T* y) {
+    const int row = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
+    const int lane = threadIdx.x % 32;
+    if (row >= M) return;
+    const float* xr = x + (long long)row * D;
+    const long long mo = (long long)(row / rows_per_seq) * mod_stride;
+    const float invD = 1.f / (float)D;
+    if (VPL > 0) {
+        float4 v[VPL > 0 ? VPL : 1];
+        float s = 0.f;
+#pragma unroll
+        for (int i = 0; i < VPL; ++i) {
+            v[i] = reinterpret_cast<const float4*>(xr)[i * 32 + lane];
+            s += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+        }
+        const float mu = free_warp_sum(s) * invD;
+        float q = 0.f;
+#pragma unroll
+        for (int i = 0; i < VPL; ++i) {
+            float a = v[i].x - mu, b = v[i].y - mu, c = v[i].z - mu, d = v[i].w - mu;
+            q += (a * a + b * b) + (c * c + d * d);
+        }
+        const float rstd = rsqrtf(free_warp_sum(q) * invD + 1e-6f);
+#pragma unroll
+        for (int i = 0; i < VPL; ++i) {
+            const int c0 = (i * 32 + lane) * 4;
+            const float4 sh = *reinterpret_cast<const float4*>(shift + mo + c0);
+            const float4 sc = *reinterpret_cast<const float4*>(scale + mo + c0);
+            float o0 = (v[i].x - mu) * rstd * (1.f + sc.x) + sh.x;
+            float o1 = (v[i].y - mu) * rstd * (1.f + sc.y) + sh.y;
+            float o2 = (v[i].z - mu) * rstd * (1.f + sc.z) + sh.z;
+            float o3 = (v[i].w - mu) * rstd * (1.f + sc.w) + sh.w;
+            if (sizeof(T) == 4) {
+                reinterpret_cast<float4*>(y + (long long)row * D)[i * 32 + lane] = make_float4(o0, o1, o2, o3);
+            } else {
+                __nv_bfloat162 lo = __floats2bfloat162_rn(o0, o1), hi = __floats2bfloat162_rn(o2, o3);
+                uint2 pk;
+                pk.x = *reinterpret_cast<uint32_t*>(&lo);
+                pk.y = *reinterpret_cast<uint32_t*>(&hi);
+                reinterpret_cast<uint2*>(y + (long long)row * D)[i * 32 + lane] = pk;
+            }
+        }
+    } else {
+        float s = 0.f;
+        for (int c = lane; c < D; c += 32) s += xr[c];
+        const float mu = free_warp_sum(s) * invD;
+        float q = 0.f;
+        for (int c = lane; c < D; c += 32) { float a = xr[c] - mu; q += a * a; }
+        const float rstd = rsqrtf(free_warp_sum(q) * invD + 1e-6f);
+        for (int c = lane; c < D; c += 32)
+            store_act(y + (long long)row * D + c, (xr[c] - mu) * rstd * (1.f + scale[mo + c]) + shift[mo + c]);
+    }
+}
+
+template <typename T>
+__global__ void convert_kernel(long long n, const float* x, T* y) {
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+        store_act(y + i, x[i]);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Tail of the pass.  For latent element (state, c, y, x): the head's token (y/p, x/p) holds the value at
+// vector position ((y%p) p + x%p) c_out + c; the first C channels are the noise prediction.  Guidance:
+// eps = eps_u + w (eps_c - eps_u).  mean = coef_x[t] x - coef_eps[t] eps.  Optionally draws the next
+// state sample = mean + sqrt(sigma2[t]) noise (drafter step / target step of the sampling loop).
+struct TailArgs {
+    int n_states, G, C, H, W, p, c_out, N_sched;
+    float cfg_scale;
+    const float* head_out; const float* x_in; long long x_stride;
+    const int32_t* t_idx; const float *coef_x, *coef_eps, *sigma2;
+    float* mean_out; long long mean_stride;
+    float* eps_out; long long eps_stride;
+    const float* noise; long long noise_stride;
+    float* sample_out; long long sample_stride;
+    float* sample_out2; long long sample2_stride; const int32_t* sample2_mask;
+};
+
+__global__ void __launch_bounds__(256) head_to_mean_kernel(TailArgs a) {
+    const int d = a.C * a.H * a.W;
+    const int gw = a.W / a.p, n_tok = (a.H / a.p) * gw, od = a.p * a.p * a.c_out;
+    const long long total = (long long)a.n_states * d;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const int st = (int)(i / d), e = (int)(i % d);
+        const int c = e / (a.H * a.W), yy = (e / a.W) % a.H, xx = e % a.W;
+        const int tok = (yy / a.p) * gw + xx / a.p;
+        const int vec = ((yy % a.p) * a.p + xx % a.p) * a.c_out + c;
+        float eps = a.head_out[((long long)(st * a.G) * n_tok + tok) * od + vec];
+        if (a.G == 2) {
+            const float eu = a.head_out[((long long)(st * a.G + 1) * n_tok + tok) * od + vec];
+            eps = eu + a.cfg_scale * (eps - eu);
+        }
+        int t = a.t_idx[st];
+        t = t < 0 ? 0 : (t >= a.N_sched ? a.N_sched - 1 : t);
+        const float xv = a.x_in[(long long)st * a.x_stride + e];
+        const float mean = a.coef_x[t] * xv - a.coef_eps[t] * eps;
+        if (a.mean_out) a.mean_out[(long long)st * a.mean_stride + e] = mean;
+        if (a.eps_out) a.eps_out[(long long)st * a.eps_stride + e] = eps;
+        if (a.noise) {
+            const float smp = mean + sqrtf(fmaxf(a.sigma2[t], 0.f)) * a.noise[(long long)st * a.noise_stride + e];
+            if (a.sample_out) a.sample_out[(long long)st * a.sample_stride + e] = smp;
+            if (a.sample_out2 && (!a.sample2_mask || a.sample2_mask[st])) a.sample_out2[(long long)st * a.sample2_stride + e] = smp;
+        }
+    }
+}
+
+}  // namespace
+
+int cond_setup(int dtype, int n_states, int G, int freq_dim, int n_classes, int N_sched,
+               const int32_t* t_idx, const int32_t* labels, const float* t_embed_value,
+               void* temb, int32_t* lab_seq, cudaStream_t s) {
+    const int S = n_states * G;
+    if (dtype == FREE_FP32)
+        cond_setup_kernel<float><<<S, 128, 0, s>>>(n_states, G, freq_dim, n_classes, N_sched, t_idx, labels, t_embed_value, (float*)temb, lab_seq);
+    else
+        cond_setup_kernel<__nv_bfloat16><<<S, 128, 0, s>>>(n_states, G, freq_dim, n_classes, N_sched, t_idx, labels, t_embed_value, (__nv_bfloat16*)temb, lab_seq);
+    return free_check_launch();
+}
+
+int patch_embed(int out_dtype, int n_states, int G, int C, int H, int W, int p, int D,
+                const float* x_in, long long x_stride, const float* pe_w, const float* pe_b, const float* pos,
+                void* out, cudaStream_t s) {
+    const int n_tok = (H / p) * (W / p);
+    const size_t smem = (size_t)C * p * p * sizeof(float);
+    const unsigned grid = (unsigned)(n_states * n_tok);
+    if (out_dtype == FREE_FP32)
+        patch_embed_kernel<float><<<grid, 128, smem, s>>>(G, C, H, W, p, D, x_in, x_stride, pe_w, pe_b, pos, (float*)out);
+    else
+        patch_embed_kernel<__nv_bfloat16><<<grid, 128, smem, s>>>(G, C, H, W, p, D, x_in, x_stride, pe_w, pe_b, pos, (__nv_bfloat16*)out);
+    return free_check_launch();
+}
+
+template <typename T>
+static int ln_launch(int M, int D, int rps, const float* x, const float* sh, const float* sc, long long ms, T* y, cudaStream_t s) {
+    const int rows_per_cta = 8;
+    const unsigned grid = (unsigned)((M + rows_per_cta - 1) / rows_per_cta);
+    const bool vec = (D % 128 == 0) && (ms % 4 == 0) && free_aligned16(sh) && free_aligned16(sc) && free_aligned16(x) && free_aligned16(y);
+    const int vpl = vec ? D / 128 : 0;
+    switch (vpl) {
+        case 3: ln_modulate_kernel<T, 3><<<grid, 256, 0, s>>>(M, D, rps, x, sh, sc, ms, y); break;    // D = 384
+        case 9: ln_modulate_kernel<T, 9><<<grid, 256, 0, s>>>(M, D, rps, x, sh, sc, ms, y); break;    // D = 1152
+        default: ln_modulate_kernel<T, 0><<<grid, 256, 0, s>>>(M, D, rps, x, sh, sc, ms, y); break;
+    }
+    return free_check_launch();
+}
+
+int ln_modulate(int out_dtype, int M, int D, int rows_per_seq, const float* x, const float* shift, const float* scale,
+                long long mod_stride, void* y, cudaStream_t s) {
+    if (M < 1 || D < 1 || rows_per_seq < 1 || !x || !shift || !scale || !y) return FREE_ERR_ARG;
+    return out_dtype == FREE_FP32 ? ln_launch<float>(M, D, rows_per_seq, x, shift, scale, mod_stride, (float*)y, s)
+                                  : ln_launch<__nv_bfloat16>(M, D, rows_per_seq, x, shift, scale, mod_stride, (__nv_bfloat16*)y, s);
+}
+
+int convert_rows(int out_dtype, long long n, const float* x, void* y, cudaStream_t s) {
+    const unsigned grid = (unsigned)((n + 255) / 256 > 148 * 16 ? 148 * 16 : (n + 255) / 256);
+    if (out_dtype == FREE_FP32) convert_kernel<float><<<grid, 256, 0, s>>>(n, x, (float*)y);
+    else convert_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(n, x, (__nv_bfloat16*)y);
+    return free_check_launch();
+}
+
+int head_to_mean(int n_states, int G, int C, int H, int W, int p, int c_out, float cfg_scale, int N_sched,
+                 const float* head_out, const float* x_in, long long x_stride,
+                 const int32_t* t_idx, const float* coef_x, const float* coef_eps, const float* sigma2,
+                 float* mean_out, long long mean_stride, float* eps_out, long long eps_stride,
+                 const float* noise, long long noise_stride, float* sample_out, long long sample_stride,
+                 float* sample_out2, long long sample2_stride, const int32_t* sample2_mask, cudaStream_t s) {
+    TailArgs a{n_states, G, C, H, W, p, c_out, N_sched, cfg_scale, head_out, x_in, x_stride, t_idx, coef_x, coef_eps, sigma2,
+               mean_out, mean_stride, eps_out, eps_stride, noise, noise_stride, sample_out, sample_stride,
+               sample_out2, sample2_stride, sample2_mask};
+    const long long total = (long long)n_states * C * H * W;
+    const unsigned grid = (unsigned)((total + 255) / 256 > 148 * 8 ? 148 * 8 : (total + 255) / 256);
+    head_to_mean_kernel<<<grid, 256, 0, s>>>(a);
+    return free_check_launch();
+}
+
+extern "C" int free_op_ln_modulate(int out_dtype, int M, int D, int rows_per_seq, const float* x,
+                                   const float* shift, const float* scale, int64_t mod_stride, void* y, void* stream) {
+    if (out_dtype != FREE_FP32 && out_dtype != FREE_BF16) return FREE_ERR_ARG;
+    return ln_modulate(out_dtype, M, D, rows_per_seq, x, shift, scale, mod_stride, y, reinterpret_cast<cudaStream_t>(stream));
+}
