@@ -220,7 +220,7 @@ int sample_trajectory(free_ctx* ctx, int B,
 /* out[M, N] = epilogue(A[M, K] * W[N, K]^T + bias[N]).  A, W in `dtype`; bias fp32 or NULL.
  * out_dtype FREE_FP32 or FREE_BF16 (ignored for GATE_RESIDUAL, whose output is the fp32 `resid`).
  * gate: DEVICE fp32, element (seq, n) at gate[seq * gate_stride + n].
- * BF16 path (tcgen05): K % 64 == 0, N % 16 == 0; FP32 path (CUDA cores): any sizes.
+ * BF16 path (tcgen05): K % 64 == 0, N % 32 == 0; FP32 path (CUDA cores): any sizes.
  * `ws` (>= free_op_linear_workspace_bytes()) holds the device error word of the pipeline. */
 size_t free_op_linear_workspace_bytes(void);
 int free_op_linear(int dtype, int epilogue, int out_dtype, int M, int N, int K,

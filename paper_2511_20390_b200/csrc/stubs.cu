@@ -1,7 +1,5 @@
 // Tensor-core kernels not written yet: report "unsupported" so that callers fail loudly.
 #include "internal.h"
-int linear_bf16(const LinearArgs&, cudaStream_t) { return FREE_ERR_UNSUPPORTED; }
-bool linear_bf16_supported(int, int) { return false; }
 int attention_tc(int, int, int, int, int, const void*, const void*, const void*, void*, uint32_t*, cudaStream_t) { return FREE_ERR_UNSUPPORTED; }
 bool attention_tc_supported(int, int) { return false; }
 int attention_tc_dpad(int d) { return d; }
