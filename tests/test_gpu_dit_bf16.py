@@ -1,0 +1,95 @@
+"""bf16 tensor-core mode against the fp64 oracle on bf16-representable weights.
+Tolerance 2e-2 = max error / max |oracle| per output tensor (the bound the task fixes for bf16)."""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle import dit as odit, drafter as odrafter, schedule as osched
+from gpu_util import cu, nerr
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-2
+
+
+@pytest.fixture(scope="module")
+def free():
+    import paper_2511_20390_b200 as f
+    f.lib()
+    return f
+
+
+def _model(free, sh, seed, depth=None, **kw):
+    import dataclasses
+    if depth is not None:
+        sh = dataclasses.replace(sh, depth=depth)
+    w = synth.make_target_weights(sh, seed, bf16=True, **kw)
+    wd = synth.make_drafter_weights(sh, seed + 1, bf16=True, **kw)
+    return sh, w, wd, free.Model(sh, w, wd, dtype="bf16")
+
+
+@pytest.mark.parametrize("kw", [dict(), dict(ada_std=0.2, out_gain=2.0)])
+def test_dit_s2_packed_pass(free, kw):
+    # DiT-S/2 shaped: 4x32x32 latents (256 tokens), width 384, 12 blocks, 6 heads; B = 4 samples x K = 6 states
+    sh, w, wd, model = _model(free, synth.DIT_S2, 11, **kw)
+    N = 250
+    sc = osched.make("respaced", N)
+    dsched = free.DeviceSchedule(free.respaced_schedule(N))
+    x, t, y = synth.pack_states(5, 4, 6, (sh.C, sh.H, sh.W), N, sh.n_classes)
+    X, T, Y = x.reshape(24, sh.C, sh.H, sh.W), t.reshape(-1), y.reshape(-1)
+    mean, eps, feat = model.dit_verify_pass(cu(X), cu(T, torch.int32), cu(Y, torch.int32), 0.0, dsched, want_eps=True, want_feat=True)
+    torch.cuda.synchronize()
+    pick = [0, 7, 13, 23]
+    mo, eo, fo = odit.verify_pass(w, sh, sc, X[pick], T[pick], Y[pick], 0.0)
+    errs = (nerr(eps[pick], eo), nerr(mean[pick], mo), nerr(feat[pick], fo))
+    print("S/2 errors eps/mean/feat:", errs)
+    assert max(errs) < TOL
+
+
+def test_dit_s2_guided_and_drafter(free):
+    sh, w, wd, model = _model(free, synth.DIT_S2, 21, depth=4, ada_std=0.2, out_gain=2.0)
+    N = 250
+    sc = osched.make("respaced", N)
+    dsched = free.DeviceSchedule(free.respaced_schedule(N))
+    n = 3
+    x = synth.normal(8, 1, (n, sh.C, sh.H, sh.W))
+    t, y = np.array([240, 100, 7], np.int32), np.array([1, 999, 400], np.int32)
+    mean, eps, feat = model.dit_verify_pass(cu(x), cu(t, torch.int32), cu(y, torch.int32), 4.0, dsched, want_eps=True, want_feat=True)
+    mo, eo, fo = odit.verify_pass(w, sh, sc, x, t, y, 4.0)
+    assert max(nerr(eps, eo), nerr(mean, mo), nerr(feat, fo)) < TOL
+    # drafter step from the oracle's features (rounded to bf16, as the GPU stores them)
+    f_prev = synth.round_to_bf16(fo.astype(np.float32))
+    z = synth.normal(8, 3, (n, sh.C, sh.H, sh.W))
+    t2 = (t - 1).astype(np.int32)
+    m_hat, x_hat, f_next = model.draft_step(cu(x), cu(f_prev, torch.bfloat16), cu(t2, torch.int32), cu(y, torch.int32), 4.0, dsched, cu(z))
+    torch.cuda.synchronize()
+    for i in range(n):
+        mo_i, eo_i, fo_i = odrafter.guided_step(w, wd, sh, sc, x[i], f_prev[i], int(t2[i]), int(y[i]), 4.0)
+        assert nerr(m_hat[i], mo_i) < TOL and nerr(f_next[i], fo_i) < TOL
+        assert nerr(x_hat[i], mo_i + np.sqrt(sc.sigma2[t2[i]]) * z[i]) < TOL
+
+
+def test_bf16_trajectory_teacher_forced(free):
+    # the sampling loop in bf16 mode on a small model: every round's decisions must be the oracle verifier's
+    # decisions on the GPU's own means; checked through the final statistics of an all-accept and an all-reject run
+    import dataclasses
+    sh = dataclasses.replace(synth.DIT_S2, depth=2, H=16, W=16)
+    N, K, B = 12, 3, 2
+    dsched = free.DeviceSchedule(free.respaced_schedule(N))
+    shape = (sh.C, sh.H, sh.W)
+    x0 = synth.normal(4, 1, (B,) + shape)
+    zt, zd = synth.normal(4, 2, (B, N) + shape), synth.normal(4, 3, (B, N) + shape)
+    labels = cu(np.array([3, 7], np.int32), torch.int32)
+    w = synth.make_target_weights(sh, 1, bf16=True)
+    wd = synth.make_drafter_weights(sh, 2, bf16=True)
+    model = free.Model(sh, w, wd, dtype="bf16")
+    # u = 0 accepts everything: rounds advance K+1 transitions
+    xf, st = model.sample_trajectory(cu(x0), labels, dsched, K, 0.0, cu(zt), cu(zd), cu(np.zeros((B, N), np.float32)))
+    assert st["rejected"] == 0 and st["accepted"] == st["draft_calls"] and torch.isfinite(xf).all()
+    assert st["parallel_efficiency"] > 1.5
+    # u = 1 with a random drafter rejects (almost) every first draft: two transitions per round
+    xf2, st2 = model.sample_trajectory(cu(x0), labels, dsched, K, 0.0, cu(zt), cu(zd), cu(np.ones((B, N), np.float32)))
+    assert st2["rejected"] >= st2["rounds"] // 2 and torch.isfinite(xf2).all()
+    # K = 0: plain sampler, N target calls per sample
+    xf3, st3 = model.sample_trajectory(cu(x0), labels, dsched, 0, 0.0, cu(zt))
+    assert st3["target_calls"] == B * N
