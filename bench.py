@@ -24,7 +24,7 @@ sys.path.insert(0, ROOT)
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--workload", default="default")
@@ -236,12 +236,16 @@ def main():
     sampler = ClockSampler(local_rank) if rank == 0 else None
     stream = torch.cuda.current_stream()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if hasattr(wl, "begin_timed"):
+        wl.begin_timed()          # per-kernel CUDA events on the launching stream, inside the timed region
     ev0.record(stream)
     for _ in range(args.steps):
         wl.step()
     ev1.record(stream)
     barrier()
     ms = ev0.elapsed_time(ev1)
+    if hasattr(wl, "end_timed"):
+        wl.end_timed(args.steps)
     kernel_ms = wl.kernel_ms_per_launch() if hasattr(wl, "kernel_ms_per_launch") else ms / args.steps
     clocks = sampler.stop() if sampler else None
 
@@ -272,7 +276,7 @@ def main():
                "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic", "config": wl.config,
                "clocks": clocks,
                "e2e": {"value": e2e_value, "unit": wl.unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-               "gpu_launches": wl.launches_per_step * args.steps,
+               "gpu_launches": int(round(wl.launches_per_step * args.steps)),
                "roofline": wl.roofline(kernel_ms, peaks)}
         if hasattr(wl, "extra"):
             out.update(wl.extra(ms_step, peaks))

@@ -1,0 +1,162 @@
+"""The benchmark's main workload: one speculative round of FREE on a DiT-XL/2-shaped model at 512^2.
+
+Step = the whole hot path once for a batch of B images (Algorithm 1's loop body): target step on the B current
+latents, K = 6 drafter steps, ONE packed target pass over B*K states (each doubled by classifier-free guidance),
+the fused verifier, the cursor update.  Weights are random-init (no checkpoints exist here), latents N(0,1),
+labels uniform over 1000 classes, 250-step respaced DDPM schedule.
+"""
+import os
+import time
+
+import numpy as np
+
+K_DRAFTS, CFG, N_SCHED = 6, 4.0, 250
+
+
+def round_flops(shape, B, K, G, n_draft_blocks=1):
+    """Algorithmic FLOPs of one round: 2MNK per linear layer + 4 T^2 d_head per (head, block, sequence);
+    target step (B*G sequences), K drafter steps (fusion layer + blocks), packed pass (B*K*G sequences)."""
+    seq = shape.flops_per_sequence()
+    fuse = 2.0 * shape.n_tok * shape.D * 2 * shape.D
+    draft = shape.flops_per_sequence(depth=n_draft_blocks) + fuse
+    return B * G * seq + K * B * G * draft + B * K * G * seq
+
+
+class RoundWorkload:
+    metric = "DiT-XL/2 512^2 packed-verify TFLOP/s"
+    unit = "TFLOP/s"
+    dtype = "bf16"
+
+    def __init__(self, batch, rank):
+        import torch
+        import synth
+        import paper_2511_20390_b200 as free
+        self.torch, self.free = torch, free
+        self.shape = synth.DIT_XL2_512
+        self.B = batch or 16
+        B, K, sh = self.B, K_DRAFTS, self.shape
+        self.model = free.Model.random(sh, 1234 + rank, dtype="bf16", with_drafter=True)
+        self.sched = free.DeviceSchedule(free.respaced_schedule(N_SCHED))
+        g = torch.Generator(device="cuda")
+        g.manual_seed(99 + rank)
+        d = sh.d_latent
+        rn = lambda *s: torch.randn(*s, generator=g, device="cuda", dtype=torch.float32)
+        self.x_cur = rn(B, sh.C, sh.H, sh.W)
+        self.labels = torch.randint(0, sh.n_classes, (B,), generator=g, device="cuda", dtype=torch.int32)
+        # every step restarts from the same cursor (transition 21 of 250), so all steps do identical work
+        self.cursor = torch.full((B,), 21, dtype=torch.int32, device="cuda")
+        self.noise_t, self.noise_d = rn(B, N_SCHED, d), rn(B, N_SCHED, d)
+        self.uniforms = torch.rand(B, N_SCHED, generator=g, device="cuda", dtype=torch.float32)
+        self.x_next = torch.empty_like(self.x_cur)
+        self.cursor_next = torch.empty_like(self.cursor)
+        self.n_acc = torch.zeros(B, dtype=torch.int32, device="cuda")
+        self.G = 2
+        self.flops = round_flops(sh, B, K, self.G)
+        self.units_per_step = self.flops / 1e12
+        self.config = {"workload": f"FREE round, DiT-XL/2-shaped 512^2 (latent 4x64x64, 1024 tokens, width 1152, 28 blocks, "
+                                   f"16 heads), K={K} drafts, cfg {CFG} (doubled batch), batch {B}, 1-block drafter, "
+                                   f"{N_SCHED}-step schedule",
+                       "B": B, "K": K, "sequences_in_packed_pass": B * K * self.G,
+                       "cache": "activations per step (several GB) exceed L2"}
+        # host staging for the end-to-end path
+        pin = lambda t: torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t)
+        self.h_in = [pin(self.x_cur), pin(self.cursor), pin(self.labels)]
+        self.h_out = [torch.empty(self.x_next.shape, dtype=torch.float32, pin_memory=True),
+                      torch.empty(B, dtype=torch.int32, pin_memory=True), torch.empty(B, dtype=torch.int32, pin_memory=True)]
+        self.launches_per_step = None
+        self._prof = None
+
+    def _round(self):
+        self.model.spec_round(self.x_cur, self.cursor, self.labels, self.sched, K_DRAFTS, CFG, self.noise_t, self.noise_d,
+                              self.uniforms, x_next=self.x_next, cursor_next=self.cursor_next, n_accept=self.n_acc)
+
+    def begin_timed(self):
+        self.model.profile_begin()
+
+    def end_timed(self, steps):
+        self._prof = self.model.profile_end()
+        self.launches_per_step = sum(p["launches"] for p in self._prof) / steps
+        err = self.model.device_error()
+        if err:
+            raise RuntimeError(f"device error word {err:#x}: a bounded wait gave up, the timing is void")
+
+    def step(self):
+        self._round()
+
+    def host_step(self):
+        t = self.torch
+        self.x_cur.copy_(self.h_in[0], non_blocking=True)
+        self.cursor.copy_(self.h_in[1], non_blocking=True)
+        self.labels.copy_(self.h_in[2], non_blocking=True)
+        self._round()
+        self.h_out[0].copy_(self.x_next, non_blocking=True)
+        self.h_out[1].copy_(self.cursor_next, non_blocking=True)
+        self.h_out[2].copy_(self.n_acc, non_blocking=True)
+        h2d = sum(x.numel() * x.element_size() for x in self.h_in)
+        d2h = sum(x.numel() * x.element_size() for x in self.h_out)
+        return h2d, d2h
+
+    def kernel_ms_per_launch(self):
+        return None
+
+    def roofline(self, _ms, peaks):
+        """Dominant kernel = the tensor-core linear-layer class with the largest share of device time."""
+        lin = [p for p in self._prof if p["name"].startswith("linear")]
+        top = max(lin, key=lambda p: p["ms"])
+        per_launch_ms = top["ms"] / top["launches"]
+        ach = top["work"] / top["launches"] / 1e12 / (per_launch_ms / 1e3)
+        peak = peaks["bf16_tflops_sustained"]
+        return {"bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
+                "traffic": None, "kernel": f"linear_tc_kernel [{top['name']}]", "launches": top["launches"],
+                "ms_per_launch": per_launch_ms, "peak_source": peaks["source"] + " (sustained bf16 GEMM)"}
+
+    def extra(self, ms_step, peaks):
+        tot = sum(p["ms"] for p in self._prof)
+        kern = []
+        for p in sorted(self._prof, key=lambda p: -p["ms"]):
+            e = {"name": p["name"], "launches": p["launches"], "ms": round(p["ms"], 3), "share": round(p["ms"] / tot, 4)}
+            if p["name"].startswith(("linear", "attention", "drafter", "head", "conditioning")) and p["ms"] > 0:
+                e["tflops"] = round(p["work"] / 1e12 / (p["ms"] / 1e3), 1)
+            elif p["work"] > 0 and p["ms"] > 0:
+                e["gbs"] = round(p["work"] / 1e9 / (p["ms"] / 1e3), 1)
+            kern.append(e)
+        value = self.flops / 1e12 / (ms_step / 1e3)
+        return {"pct_of_bf16_peak": {"of_measured_sustained": value / peaks["bf16_tflops_sustained"],
+                                     "of_measured_burst": value / peaks["bf16_tflops"], "of_nominal_2250": value / 2250.0},
+                "images_per_s_if_all_accepted": self.B * (K_DRAFTS + 1) / N_SCHED / (ms_step / 1e3),
+                "kernels": kern}
+
+    def oracle_sample(self):
+        return oracle_dit_sample(self.shape)
+
+
+def oracle_dit_sample(shape, n_blocks=3):
+    """Times the fp64 oracle on one sequence through `n_blocks` of the 28 blocks (plus embedding and head)."""
+    import dataclasses
+    import synth
+    from oracle import dit as odit
+    sh = dataclasses.replace(shape, depth=n_blocks)
+    w = synth.make_target_weights(sh, 5, bf16=True)
+    x = synth.normal(5, 77, (sh.C, sh.H, sh.W))
+    t0 = time.perf_counter()
+    odit.forward(w, sh, x, 500.0, 7)
+    dt = time.perf_counter() - t0
+    return sh.flops_per_sequence() / 1e12 / dt, f"1 sequence (1024 tokens) through {n_blocks} of 28 blocks, fp64 numpy"
+
+
+def reference_arm(args, cores):
+    """bench.py --impl reference: the oracle as it stands, one bounded sample per step."""
+    import synth
+    shape = synth.DIT_XL2_512
+    vals = []
+    for _ in range(min(args.warmup, 1)):
+        oracle_dit_sample(shape, 1)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        v, sample = oracle_dit_sample(shape, 2)
+        vals.append(v)
+    dt = (time.perf_counter() - t0) / max(args.steps, 1)
+    val = float(np.mean(vals))
+    return {"metric": RoundWorkload.metric, "value": val, "unit": "TFLOP/s", "ms_per_step": dt * 1e3, "dtype": "f64",
+            "config": {"workload": "FREE round, DiT-XL/2-shaped 512^2, K=6, cfg 4, batch 16 (oracle: bounded sample)"},
+            "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample}}

@@ -9,6 +9,10 @@
  *     16-byte aligned; pointers marked HOST are ordinary host memory.  The caller owns every buffer.
  *     The library allocates no device memory: scratch space is the caller's workspace `ws`, sized by
  *     free_workspace_bytes().  Tensors are dense, row-major, innermost index last.
+ *   - Device-side waits are bounded.  If one gives up, the kernels stop early and OR a non-zero code into the
+ *     first 4 bytes of the workspace (the "device error word", cleared at the start of every call that takes a
+ *     workspace); results are then invalid.  sample_trajectory() returns FREE_ERR_DEVICE_TIMEOUT itself;
+ *     for the asynchronous calls the caller reads the word after synchronising.
  *   - `stream` is a cudaStream_t passed as void*.  Work is enqueued on it and the call returns
  *     without waiting, except sample_trajectory(), which synchronises once per round.
  *   - No random numbers are drawn inside: noise and uniforms are inputs, so that a run can be
@@ -206,6 +210,36 @@ int sample_trajectory(free_ctx* ctx, int B,
                            const float* noise_target, const float* noise_draft, const float* uniforms,
                            float* x_final, free_traj_stats* stats,
                            void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * spec_round -- the body of Algorithm 1's loop, once: for every sample b whose cursor[b] <= N (cursor = index of
+ * the next transition, 1-based), target step on x_cur[b], K drafter steps, packed target pass, verification;
+ * x_next[b] is the last finalised state and cursor_next[b] points past it.  sample_trajectory is this call
+ * repeated until every cursor exceeds N.  Asynchronous.  Arguments as for sample_trajectory;
+ *   x_cur, x_next DEVICE fp32 [B, C, H, W] (may alias); cursor, cursor_next DEVICE int32 [B] (may alias);
+ *   n_accept DEVICE int32 [B] or NULL: drafts accepted this round (undefined for samples that drafted nothing).
+ */
+int free_spec_round(free_ctx* ctx, int B, const float* x_cur, const int32_t* cursor, const int32_t* labels,
+                    const free_schedule* sched, const free_spec_params* params,
+                    const float* noise_target, const float* noise_draft, const float* uniforms,
+                    float* x_next, int32_t* cursor_next, int32_t* n_accept,
+                    void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Per-kernel timing (measurement aid; the paper has no counterpart).  Between free_profile_begin() and
+ * free_profile_end() every kernel launched by the context's passes is bracketed by CUDA events on the caller's
+ * stream.  free_profile_end() waits for them and returns one entry per kernel class: launches, summed device time
+ * and summed algorithmic work (FLOPs for linear layers and attention, bytes for the bandwidth-bound kernels).
+ * `out` is HOST memory with room for max_entries entries.
+ */
+typedef struct free_prof_entry {
+    char    name[48];
+    int64_t launches;
+    double  ms;
+    double  work;
+} free_prof_entry;
+int free_profile_begin(free_ctx* ctx);
+int free_profile_end(free_ctx* ctx, free_prof_entry* out, int max_entries, int* n_entries);
 
 /* ------------------------------------------------------------------------------------------------
  * Building blocks, exported so that each kernel can be checked against the CPU oracle on its own.

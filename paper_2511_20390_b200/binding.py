@@ -49,6 +49,10 @@ class SpecParams(C.Structure):
     _fields_ = [("K", C.c_int32), ("cfg_scale", C.c_float), ("lam", C.c_void_p)]
 
 
+class ProfEntry(C.Structure):
+    _fields_ = [("name", C.c_char * 48), ("launches", C.c_int64), ("ms", C.c_double), ("work", C.c_double)]
+
+
 class TrajStats(C.Structure):
     _fields_ = [("rounds", C.c_int64), ("target_calls", C.c_int64), ("draft_calls", C.c_int64),
                 ("accepted", C.c_int64), ("rejected", C.c_int64),
@@ -72,6 +76,11 @@ _SIGNATURES = {
     "sample_trajectory": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.POINTER(ScheduleDesc),
                                     C.POINTER(SpecParams), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                     C.POINTER(TrajStats), C.c_void_p, C.c_size_t, C.c_void_p]),
+    "free_spec_round": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(ScheduleDesc),
+                                  C.POINTER(SpecParams), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                  C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "free_profile_begin": (C.c_int, [C.c_void_p]),
+    "free_profile_end": (C.c_int, [C.c_void_p, C.POINTER(ProfEntry), C.c_int, C.POINTER(C.c_int)]),
     "free_op_linear_workspace_bytes": (C.c_size_t, []),
     "free_op_linear": (C.c_int, [C.c_int] * 6 + [C.c_void_p] * 6 + [C.c_int64, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]),
     "free_op_ln_modulate": (C.c_int, [C.c_int] * 4 + [C.c_void_p] * 3 + [C.c_int64, C.c_void_p, C.c_void_p]),
@@ -203,6 +212,10 @@ class DeviceSchedule:
 def _upload(weights: dict, dtype: int, device):
     out = {}
     for k, v in weights.items():
+        if isinstance(v, torch.Tensor):
+            t = v.to(device)
+            out[k] = (t.to(_ACT[dtype]) if k in _MATRICES else t.to(torch.float32)).contiguous()
+            continue
         t = torch.from_numpy(np.ascontiguousarray(v, dtype=np.float32)).to(device)
         out[k] = t.to(_ACT[dtype]).contiguous() if k in _MATRICES else t
     return out
@@ -257,6 +270,72 @@ class Model:
             self._ws = None
             self._ws = torch.empty(need, dtype=torch.uint8, device=self.device)
         return self._ws
+
+    @classmethod
+    def random(cls, shape, seed: int, dtype: str = "bf16", with_drafter: bool = True, n_draft_blocks: int = 1,
+               std: float = 0.02, device="cuda"):
+        """Random-init model whose weights are drawn on the device (no host copy): for timing runs, where the
+        values only need the right shapes and scale.  The fixed position table comes from `synth`."""
+        import synth
+        g = torch.Generator(device=device)
+        g.manual_seed(int(seed))
+        D, F = shape.D, shape.mlp_ratio * shape.D
+        act = _ACT[{"fp32": FREE_FP32, "bf16": FREE_BF16}[dtype]]
+
+        def mat(*s):
+            return (torch.randn(*s, generator=g, device=device, dtype=torch.float32) * std).to(act)
+
+        def vec(*s):
+            return torch.randn(*s, generator=g, device=device, dtype=torch.float32) * std
+
+        def blocks(n):
+            return {"ada_w": mat(n, 6 * D, D), "ada_b": vec(n, 6 * D), "qkv_w": mat(n, 3 * D, D), "qkv_b": vec(n, 3 * D),
+                    "proj_w": mat(n, D, D), "proj_b": vec(n, D), "fc1_w": mat(n, F, D), "fc1_b": vec(n, F),
+                    "fc2_w": mat(n, D, F), "fc2_b": vec(n, D), "fada_w": mat(2 * D, D), "fada_b": vec(2 * D),
+                    "fin_w": vec(shape.out_dim, D), "fin_b": vec(shape.out_dim)}
+        w = {"t_w1": mat(D, shape.freq_dim), "t_b1": vec(D), "t_w2": mat(D, D), "t_b2": vec(D),
+             "y_emb": vec(shape.n_classes + 1, D), "pe_w": vec(D, shape.patch_dim), "pe_b": vec(D),
+             "pos": torch.from_numpy(synth.pos_embed_2d(shape)).to(device)}
+        w.update(blocks(shape.depth))
+        wd = None
+        if with_drafter:
+            wd = {"fc_w": mat(D, 2 * D), "fc_b": vec(D)}
+            wd.update(blocks(n_draft_blocks))
+        return cls(shape, w, wd, dtype=dtype, n_draft_blocks=n_draft_blocks, device=device)
+
+    def device_error(self) -> int:
+        """The device error word of the last call that used the workspace (0 = no bounded wait gave up).
+        Synchronises the current stream."""
+        if self._ws is None:
+            return 0
+        torch.cuda.current_stream().synchronize()
+        return int(self._ws[:4].view(torch.int32).item())
+
+    def profile_begin(self):
+        _check(lib().free_profile_begin(self.ctx), "free_profile_begin")
+
+    def profile_end(self):
+        """Per-kernel-class totals since profile_begin(): list of dicts name / launches / ms / work."""
+        buf = (ProfEntry * 32)()
+        n = C.c_int(0)
+        _check(lib().free_profile_end(self.ctx, buf, 32, C.byref(n)), "free_profile_end")
+        return [{"name": buf[i].name.decode(), "launches": buf[i].launches, "ms": buf[i].ms, "work": buf[i].work}
+                for i in range(n.value)]
+
+    def spec_round(self, x_cur, cursor, labels, sched, K, cfg_scale, noise_target, noise_draft=None, uniforms=None,
+                   lam=None, x_next=None, cursor_next=None, n_accept=None):
+        """One round of Algorithm 1 (asynchronous).  Returns (x_next, cursor_next, n_accept)."""
+        B = x_cur.shape[0]
+        _dev(x_cur, torch.float32); _dev(cursor, torch.int32); _dev(labels, torch.int32)
+        prm = SpecParams(int(K), float(cfg_scale), None if lam is None else _dev(lam, torch.float32).data_ptr())
+        x_next = torch.empty_like(x_cur) if x_next is None else x_next
+        cursor_next = torch.empty_like(cursor) if cursor_next is None else cursor_next
+        n_accept = torch.zeros(B, dtype=torch.int32, device=x_cur.device) if n_accept is None else n_accept
+        ws = self.workspace(B * max(int(K), 1))
+        _check(lib().free_spec_round(self.ctx, B, _ptr(x_cur), _ptr(cursor), _ptr(labels), C.byref(sched.desc), C.byref(prm),
+                                     _ptr(noise_target), _ptr(noise_draft), _ptr(uniforms), _ptr(x_next), _ptr(cursor_next),
+                                     _ptr(n_accept), _ptr(ws), ws.numel(), _stream()), "free_spec_round")
+        return x_next, cursor_next, n_accept
 
     @staticmethod
     def guided(cfg_scale: float) -> int:

@@ -5,7 +5,19 @@
 #include <string.h>
 #include <vector>
 
+enum { PC_COND = 0, PC_EMBED, PC_LN, PC_QKV, PC_ATTN, PC_PROJ, PC_FC1, PC_FC2, PC_HEAD, PC_TAIL, PC_DRAFT_FC,
+       PC_VERIFY, PC_CTRL, PC_N };
+static const char* const kProfNames[PC_N] = {
+    "conditioning + modulation tables", "patch embed / feature copy", "layernorm + modulate", "linear qkv",
+    "attention", "linear proj (gate + residual)", "linear fc1 + gelu", "linear fc2 (gate + residual)",
+    "head (layernorm + projection)", "unpatchify + guidance + mean", "drafter fusion layer", "spec_verify",
+    "round control"};
+
+struct ProfRec { int cls; double work; cudaEvent_t e0, e1; };
+
 struct free_ctx {
+    mutable bool prof_on = false;
+    mutable std::vector<ProfRec> prof;
     free_model_desc m;
     bool has_drafter;
     free_drafter_desc dr;
@@ -15,6 +27,20 @@ struct free_ctx {
 };
 
 namespace {
+
+// Brackets one kernel launch (or a short group) with CUDA events when profiling is on.
+struct Scope {
+    const free_ctx* c; cudaStream_t s; cudaEvent_t e1 = nullptr;
+    Scope(const free_ctx* c_, int cls, double work, cudaStream_t s_) : c(c_), s(s_) {
+        if (!c->prof_on) return;
+        ProfRec r{cls, work, nullptr, nullptr};
+        if (cudaEventCreate(&r.e0) != cudaSuccess || cudaEventCreate(&r.e1) != cudaSuccess) { (void)cudaGetLastError(); return; }
+        cudaEventRecord(r.e0, s);
+        e1 = r.e1;
+        c->prof.push_back(r);
+    }
+    ~Scope() { if (e1) cudaEventRecord(e1, s); }
+};
 
 inline size_t act_size(int dtype) { return dtype == FREE_BF16 ? 2 : 4; }
 
@@ -95,6 +121,7 @@ int run_cond(const free_ctx* c, const Workspace& w, const Stack& st, int n_state
              const int32_t* t_idx, const int32_t* labels, const free_schedule* sch, cudaStream_t s) {
     const free_model_desc& m = c->m;
     const int S = n_states * G, D = m.D;
+    Scope prof(c, PC_COND, 2.0 * S * D * ((double)m.freq_dim + D + st.n_blocks * 6.0 * D + 2.0 * D), s);
     FREE_TRY(cond_setup(m.dtype, n_states, G, m.freq_dim, m.n_classes, sch->N, t_idx, labels, sch->t_embed_value,
                         w.temb, w.lab_seq, s));
     LinearArgs a;
@@ -127,7 +154,8 @@ int run_blocks(const free_ctx* c, const Workspace& w, const Stack& st, int S, cu
         const float* mod = w.mod + (size_t)i * 6 * D;
         auto wmat = [&](const void* base, size_t rows) { return (const void*)((const char*)base + (size_t)i * rows * D * as); };
         // attention branch
-        FREE_TRY(ln_modulate(m.dtype, M, D, T, w.x, mod, mod + D, ms, w.hn, s));
+        const double ln_bytes = (double)M * D * (4 + as);
+        { Scope p(c, PC_LN, ln_bytes, s); FREE_TRY(ln_modulate(m.dtype, M, D, T, w.x, mod, mod + D, ms, w.hn, s)); }
         LinearArgs a; a.err = w.err;
         a.M = M; a.N = 3 * D; a.K = D; a.A = w.hn; a.W = wmat(st.bw.qkv_w, 3 * D); a.bias = st.bw.qkv_b + (size_t)i * 3 * D;
         a.out_dtype = m.dtype;
@@ -135,27 +163,29 @@ int run_blocks(const free_ctx* c, const Workspace& w, const Stack& st, int S, cu
             a.epi = EPI_QKV_HEADS; a.heads = m.heads; a.d_head = c->d_head; a.d_pad = c->d_pad; a.n_tok = T;
             const size_t per = (size_t)S * m.heads * T * c->d_pad * 2;
             a.q = w.qkv; a.k = (char*)w.qkv + per; a.vt = (char*)w.qkv + 2 * per;
-            FREE_TRY(lin(c, a, s));
-            FREE_TRY(attention_tc(S, T, m.heads, c->d_head, c->d_pad, a.q, a.k, a.vt, w.att, w.err, s));
+            { Scope p(c, PC_QKV, 2.0 * M * 3 * D * D, s); FREE_TRY(lin(c, a, s)); }
+            { Scope p(c, PC_ATTN, 4.0 * S * m.heads * (double)T * T * c->d_head, s);
+              FREE_TRY(attention_tc(S, T, m.heads, c->d_head, c->d_pad, a.q, a.k, a.vt, w.att, w.err, s)); }
         } else {
             a.epi = EPI_BIAS; a.out = w.qkv;
-            FREE_TRY(lin(c, a, s));
-            FREE_TRY(attention_simt(m.dtype, S, T, m.heads, c->d_head, w.qkv, w.att, s));
+            { Scope p(c, PC_QKV, 2.0 * M * 3 * D * D, s); FREE_TRY(lin(c, a, s)); }
+            { Scope p(c, PC_ATTN, 4.0 * S * m.heads * (double)T * T * c->d_head, s);
+              FREE_TRY(attention_simt(m.dtype, S, T, m.heads, c->d_head, w.qkv, w.att, s)); }
         }
         a = LinearArgs(); a.err = w.err;
         a.M = M; a.N = D; a.K = D; a.A = w.att; a.W = wmat(st.bw.proj_w, D); a.bias = st.bw.proj_b + (size_t)i * D;
         a.epi = EPI_GATE_RESIDUAL; a.resid = w.x; a.gate = mod + 2 * D; a.gate_stride = ms; a.rows_per_seq = T;
-        FREE_TRY(lin(c, a, s));
+        { Scope p(c, PC_PROJ, 2.0 * M * D * D, s); FREE_TRY(lin(c, a, s)); }
         // MLP branch
-        FREE_TRY(ln_modulate(m.dtype, M, D, T, w.x, mod + 3 * D, mod + 4 * D, ms, w.hn, s));
+        { Scope p(c, PC_LN, ln_bytes, s); FREE_TRY(ln_modulate(m.dtype, M, D, T, w.x, mod + 3 * D, mod + 4 * D, ms, w.hn, s)); }
         a = LinearArgs(); a.err = w.err;
         a.M = M; a.N = F; a.K = D; a.A = w.hn; a.W = wmat(st.bw.fc1_w, F); a.bias = st.bw.fc1_b + (size_t)i * F;
         a.epi = EPI_BIAS_GELU; a.out_dtype = m.dtype; a.out = w.hmlp;
-        FREE_TRY(lin(c, a, s));
+        { Scope p(c, PC_FC1, 2.0 * M * F * D, s); FREE_TRY(lin(c, a, s)); }
         a = LinearArgs(); a.err = w.err;
         a.M = M; a.N = D; a.K = F; a.A = w.hmlp; a.W = (const char*)st.bw.fc2_w + (size_t)i * D * F * as; a.bias = st.bw.fc2_b + (size_t)i * D;
         a.epi = EPI_GATE_RESIDUAL; a.resid = w.x; a.gate = mod + 5 * D; a.gate_stride = ms; a.rows_per_seq = T;
-        FREE_TRY(lin(c, a, s));
+        { Scope p(c, PC_FC2, 2.0 * M * F * D, s); FREE_TRY(lin(c, a, s)); }
     }
     return FREE_OK;
 }
@@ -164,6 +194,7 @@ int run_blocks(const free_ctx* c, const Workspace& w, const Stack& st, int S, cu
 int run_head(const free_ctx* c, const Workspace& w, const Stack& st, int S, cudaStream_t s) {
     const free_model_desc& m = c->m;
     const int D = m.D, T = c->n_tok, M = S * T;
+    Scope prof(c, PC_HEAD, 2.0 * M * D * c->out_dim, s);
     FREE_TRY(ln_modulate(FREE_FP32, M, D, T, w.x, w.fmod, w.fmod + D, 2LL * D, w.hn, s));
     LinearArgs a;
     a.M = M; a.N = c->out_dim; a.K = D; a.A = w.hn; a.W = st.fin_w; a.bias = st.fin_b;
@@ -193,6 +224,7 @@ Stack drafter_stack(const free_ctx* c) {
 int tail(const free_ctx* c, const Workspace& w, int n_states, int G, float cfg, const free_schedule* sch,
          const PassIO& io, cudaStream_t s) {
     const free_model_desc& m = c->m;
+    Scope prof(c, PC_TAIL, (double)n_states * c->d_latent * 4 * 3, s);
     return head_to_mean(n_states, G, m.C, m.H, m.W, m.patch, m.c_out, cfg, sch->N, w.head_out, io.x_in, io.x_stride,
                         io.t_idx, sch->coef_x, sch->coef_eps, sch->sigma2, io.mean_out, io.mean_stride,
                         io.eps_out, c->d_latent, io.noise, io.noise_stride, io.sample_out, io.sample_stride,
@@ -205,9 +237,11 @@ int target_pass(const free_ctx* c, const Workspace& w, int n_states, float cfg, 
     const int G = (cfg > 0.f && cfg != 1.f) ? 2 : 1, S = n_states * G;
     const Stack st = target_stack(c);
     FREE_TRY(run_cond(c, w, st, n_states, G, io.t_idx, io.labels, sch, s));
-    FREE_TRY(patch_embed(FREE_FP32, n_states, G, m.C, m.H, m.W, m.patch, m.D, io.x_in, io.x_stride, m.pe_w, m.pe_b, m.pos, w.x, s));
+    { Scope p(c, PC_EMBED, (double)S * c->n_tok * m.D * 4, s);
+      FREE_TRY(patch_embed(FREE_FP32, n_states, G, m.C, m.H, m.W, m.patch, m.D, io.x_in, io.x_stride, m.pe_w, m.pe_b, m.pos, w.x, s)); }
     FREE_TRY(run_blocks(c, w, st, S, s));
-    if (io.feat_out) FREE_TRY(convert_rows(m.dtype, (long long)S * c->n_tok * m.D, w.x, io.feat_out, s));
+    if (io.feat_out) { Scope p(c, PC_EMBED, (double)S * c->n_tok * m.D * 6, s);
+                       FREE_TRY(convert_rows(m.dtype, (long long)S * c->n_tok * m.D, w.x, io.feat_out, s)); }
     FREE_TRY(run_head(c, w, st, S, s));
     return tail(c, w, n_states, G, cfg, sch, io, s);
 }
@@ -219,18 +253,20 @@ int drafter_pass(const free_ctx* c, const Workspace& w, int n_states, float cfg,
     const size_t as = act_size(m.dtype);
     const Stack st = drafter_stack(c);
     FREE_TRY(run_cond(c, w, st, n_states, G, io.t_idx, io.labels, sch, s));
-    FREE_TRY(patch_embed(m.dtype, n_states, G, m.C, m.H, m.W, m.patch, D, io.x_in, io.x_stride, m.pe_w, m.pe_b, m.pos, w.emb, s));
+    { Scope p(c, PC_EMBED, (double)M * D * as, s);
+      FREE_TRY(patch_embed(m.dtype, n_states, G, m.C, m.H, m.W, m.patch, D, io.x_in, io.x_stride, m.pe_w, m.pe_b, m.pos, w.emb, s)); }
+    Scope* fc = new Scope(c, PC_DRAFT_FC, 2.0 * M * D * 2 * D, s);
     // g = W_fc [embed || f] + b  as two accumulating GEMMs over the two halves of W_fc (row stride 2D)
     LinearArgs a; a.err = w.err;
     a.M = M; a.N = D; a.K = D; a.A = w.emb; a.W = c->dr.fc_w; a.ldw = 2 * D; a.bias = c->dr.fc_b;
     a.epi = EPI_BIAS; a.out_dtype = FREE_FP32; a.out = w.x;
-    FREE_TRY(lin(c, a, s));
+    { const int r1 = lin(c, a, s); if (r1 != FREE_OK) { delete fc; return r1; } }
     a = LinearArgs(); a.err = w.err;
     a.M = M; a.N = D; a.K = D; a.A = f_prev; a.W = (const char*)c->dr.fc_w + (size_t)D * as; a.ldw = 2 * D;
     a.epi = EPI_GATE_RESIDUAL; a.resid = w.x; a.gate = nullptr; a.rows_per_seq = c->n_tok;
-    FREE_TRY(lin(c, a, s));
+    { const int r2 = lin(c, a, s); delete fc; FREE_TRY(r2); }
     FREE_TRY(run_blocks(c, w, st, S, s));
-    if (io.feat_out) FREE_TRY(convert_rows(m.dtype, (long long)M * D, w.x, io.feat_out, s));
+    if (io.feat_out) { Scope p(c, PC_EMBED, (double)M * D * 6, s); FREE_TRY(convert_rows(m.dtype, (long long)M * D, w.x, io.feat_out, s)); }
     FREE_TRY(run_head(c, w, st, S, s));
     return tail(c, w, n_states, G, cfg, sch, io, s);
 }
@@ -393,6 +429,7 @@ extern "C" int dit_verify_pass(free_ctx* c, int n_states, const float* x_in, con
     FREE_TRY(check_common(c, n_states, sch, ws, ws_bytes));
     if (!free_aligned16(x_in) || !free_aligned16(mean_out) || !free_aligned16(eps_out) || !free_aligned16(feat_out)) return FREE_ERR_ALIGN;
     const Workspace w = plan(c, n_states, ws);
+    FREE_CUDA_TRY(cudaMemsetAsync(w.err, 0, 4, reinterpret_cast<cudaStream_t>(stream)));
     PassIO io{};
     io.x_in = x_in; io.x_stride = c->d_latent; io.t_idx = t_idx; io.labels = labels;
     io.mean_out = mean_out; io.mean_stride = c->d_latent; io.eps_out = eps_out; io.feat_out = feat_out;
@@ -408,6 +445,7 @@ extern "C" int draft_step(free_ctx* c, int n_states, const float* x_prev, const 
     if (!free_aligned16(x_prev) || !free_aligned16(f_prev) || !free_aligned16(noise) || !free_aligned16(m_hat) ||
         !free_aligned16(x_hat) || !free_aligned16(f_next)) return FREE_ERR_ALIGN;
     const Workspace w = plan(c, n_states, ws);
+    FREE_CUDA_TRY(cudaMemsetAsync(w.err, 0, 4, reinterpret_cast<cudaStream_t>(stream)));
     PassIO io{};
     io.x_in = x_prev; io.x_stride = c->d_latent; io.t_idx = t_idx; io.labels = labels;
     io.mean_out = m_hat; io.mean_stride = c->d_latent; io.feat_out = f_next;
@@ -415,77 +453,134 @@ extern "C" int draft_step(free_ctx* c, int n_states, const float* x_prev, const 
     return drafter_pass(c, w, n_states, cfg_scale, sch, io, f_prev, reinterpret_cast<cudaStream_t>(stream));
 }
 
+namespace {
+
+struct RoundIO {
+    int B, K;
+    const int32_t* labels;
+    const free_schedule* sch;
+    float cfg;
+    const float* lambda;
+    const float *noise_target, *noise_draft, *uniforms;
+};
+
+// One round of Algorithm 1 for every sample whose cursor has not passed N: target step, K drafter steps,
+// packed target pass, verification, cursor update.  State (w.x_cur, w.cur_a) lives in the workspace.
+int one_round(const free_ctx* c, const Workspace& w, const RoundIO& r, cudaStream_t s) {
+    const int B = r.B, K = r.K, N = r.sch->N, d = c->d_latent;
+    const free_schedule* sch = r.sch;
+    RoundArgs ra{B, K, N, r.labels, sch->sigma2, r.lambda, r.uniforms, w.cur_a, w.nv, w.t_step, w.t_pack, w.lab_pack,
+                 w.t_draft, w.act_draft, w.active, w.sigma2_bk, w.lam_bk, w.u_bk};
+    const unsigned egrid = (unsigned)(((long long)B * d + 255) / 256 > 148 * 8 ? 148 * 8 : ((long long)B * d + 255) / 256);
+    { Scope p(c, PC_CTRL, 0, s);
+      round_setup_kernel<<<(B + 127) / 128, 128, 0, s>>>(ra);
+      FREE_TRY(free_check_launch()); }
+    // (1) target step on the current state of every sample
+    PassIO io{};
+    io.x_in = w.x_cur; io.x_stride = d; io.t_idx = w.t_step; io.labels = r.labels;
+    io.mean_out = w.m_a; io.mean_stride = d; io.feat_out = K > 0 ? w.feat0 : nullptr;
+    FREE_TRY(target_pass(c, w, B, r.cfg, sch, io, s));
+    { Scope p(c, PC_CTRL, 0, s);
+      target_sample_kernel<<<egrid, 256, 0, s>>>(B, K, d, N, w.cur_a, w.active, w.t_step, sch->sigma2, w.m_a,
+                                                  r.noise_target, w.x_cur, w.pack_in);
+      FREE_TRY(free_check_launch()); }
+    if (K > 0) {
+        // (2) K drafter steps, each from the previous draft and feature
+        void* f_prev = w.feat0; void* f_next = w.feat1;
+        for (int i = 0; i < K; ++i) {
+            PassIO di{};
+            di.x_in = w.pack_in + (size_t)i * d; di.x_stride = (long long)K * d;         // x_hat_{a+i}
+            di.t_idx = w.t_draft + (size_t)i * B; di.labels = r.labels;
+            di.mean_out = w.m_draft + (size_t)i * d; di.mean_stride = (long long)K * d;
+            di.feat_out = f_next;
+            FREE_TRY(drafter_pass(c, w, B, r.cfg, sch, di, f_prev, s));
+            { Scope p(c, PC_CTRL, 0, s);
+              draft_sample_kernel<<<egrid, 256, 0, s>>>(B, K, d, N, i, w.cur_a, w.t_draft + (size_t)i * B, sch->sigma2,
+                                                         w.m_draft, r.noise_draft, w.x_draft, w.pack_in);
+              FREE_TRY(free_check_launch()); }
+            void* tmp = f_prev; f_prev = f_next; f_next = tmp;
+        }
+        // (3) one packed target pass over (x_a, x_hat_{a+1..a+K-1}) -> m_{a+1..a+K}
+        PassIO pi{};
+        pi.x_in = w.pack_in; pi.x_stride = d; pi.t_idx = w.t_pack; pi.labels = w.lab_pack;
+        pi.mean_out = w.m_target; pi.mean_stride = d;
+        FREE_TRY(target_pass(c, w, B * K, r.cfg, sch, pi, s));
+        // (4) sequential verification with the first-rejection break; the finalised state replaces x_cur
+        { Scope p(c, PC_VERIFY, (double)B * (3.0 * K + 1) * d * 4, s);
+          FREE_TRY(spec_verify(B, K, d, w.m_target, w.m_draft, w.x_draft, w.sigma2_bk, w.lam_bk, w.u_bk, w.nv,
+                               w.x_cur, w.n_acc, nullptr, s)); }
+    }
+    Scope p(c, PC_CTRL, 0, s);
+    cursor_update_kernel<<<(B + 127) / 128, 128, 0, s>>>(B, w.active, w.nv, w.n_acc, w.cur_a);
+    return free_check_launch();
+}
+
+int check_round_args(const free_ctx* c, int B, int K, const free_schedule* sch, void* ws, size_t ws_bytes,
+                     const float* noise_draft, const float* uniforms) {
+    if (B < 1) return FREE_ERR_SHAPE;
+    if (K < 0 || K > FREE_MAX_K) return FREE_ERR_SHAPE;
+    if (K > 0 && (!noise_draft || !uniforms)) return FREE_ERR_ARG;
+    FREE_TRY(check_common(c, B * (K > 0 ? K : 1), sch, ws, ws_bytes));
+    if (K > 0 && !c->has_drafter) return FREE_ERR_ARG;
+    return FREE_OK;
+}
+
+}  // namespace
+
+extern "C" int free_spec_round(free_ctx* c, int B, const float* x_cur, const int32_t* cursor, const int32_t* labels,
+                               const free_schedule* sch, const free_spec_params* prm,
+                               const float* noise_target, const float* noise_draft, const float* uniforms,
+                               float* x_next, int32_t* cursor_next, int32_t* n_accept,
+                               void* ws, size_t ws_bytes, void* stream) {
+    if (!x_cur || !cursor || !labels || !prm || !noise_target || !x_next || !cursor_next) return FREE_ERR_ARG;
+    FREE_TRY(check_round_args(c, B, prm->K, sch, ws, ws_bytes, noise_draft, uniforms));
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const int K = prm->K, d = c->d_latent;
+    const Workspace w = plan(c, B * (K > 0 ? K : 1), ws);
+    FREE_CUDA_TRY(cudaMemsetAsync(w.err, 0, 4, s));
+    FREE_CUDA_TRY(cudaMemcpyAsync(w.x_cur, x_cur, (size_t)B * d * 4, cudaMemcpyDeviceToDevice, s));
+    FREE_CUDA_TRY(cudaMemcpyAsync(w.cur_a, cursor, (size_t)B * 4, cudaMemcpyDeviceToDevice, s));
+    RoundIO r{B, K, labels, sch, prm->cfg_scale, prm->lambda, noise_target, noise_draft, uniforms};
+    FREE_TRY(one_round(c, w, r, s));
+    FREE_CUDA_TRY(cudaMemcpyAsync(x_next, w.x_cur, (size_t)B * d * 4, cudaMemcpyDeviceToDevice, s));
+    FREE_CUDA_TRY(cudaMemcpyAsync(cursor_next, w.cur_a, (size_t)B * 4, cudaMemcpyDeviceToDevice, s));
+    if (n_accept && K > 0) FREE_CUDA_TRY(cudaMemcpyAsync(n_accept, w.n_acc, (size_t)B * 4, cudaMemcpyDeviceToDevice, s));
+    return FREE_OK;
+}
+
 extern "C" int sample_trajectory(free_ctx* c, int B, const float* x0, const int32_t* labels, const free_schedule* sch,
                                  const free_spec_params* prm, const float* noise_target, const float* noise_draft,
                                  const float* uniforms, float* x_final, free_traj_stats* stats,
                                  void* ws, size_t ws_bytes, void* stream) {
     if (!x0 || !labels || !prm || !noise_target || !x_final) return FREE_ERR_ARG;
-    if (B < 1) return FREE_ERR_SHAPE;
+    FREE_TRY(check_round_args(c, B, prm->K, sch, ws, ws_bytes, noise_draft, uniforms));
     const int K = prm->K;
-    if (K < 0 || K > FREE_MAX_K) return FREE_ERR_SHAPE;
-    if (K > 0 && (!noise_draft || !uniforms)) return FREE_ERR_ARG;
-    const int n_plan = B * (K > 0 ? K : 1);
-    FREE_TRY(check_common(c, n_plan, sch, ws, ws_bytes));
-    if (K > 0 && !c->has_drafter) return FREE_ERR_ARG;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    const Workspace w = plan(c, n_plan, ws);
+    const Workspace w = plan(c, B * (K > 0 ? K : 1), ws);
     const int N = sch->N, d = c->d_latent;
-    const float cfg = prm->cfg_scale;
     if (stats) memset(stats, 0, sizeof(*stats));
 
+    FREE_CUDA_TRY(cudaMemsetAsync(w.err, 0, 4, s));
     FREE_CUDA_TRY(cudaMemcpyAsync(w.x_cur, x0, (size_t)B * d * 4, cudaMemcpyDeviceToDevice, s));
     fill_i32_kernel<<<(B + 127) / 128, 128, 0, s>>>(B, 1, w.cur_a);
+    FREE_TRY(free_check_launch());
     std::vector<int32_t> h_a(B, 1), h_nv(B), h_acc(B), h_act(B);
-    RoundArgs ra{B, K, N, labels, sch->sigma2, prm->lambda, uniforms, w.cur_a, w.nv, w.t_step, w.t_pack, w.lab_pack,
-                 w.t_draft, w.act_draft, w.active, w.sigma2_bk, w.lam_bk, w.u_bk};
-    const unsigned egrid = (unsigned)(((long long)B * d + 255) / 256 > 148 * 8 ? 148 * 8 : ((long long)B * d + 255) / 256);
+    RoundIO r{B, K, labels, sch, prm->cfg_scale, prm->lambda, noise_target, noise_draft, uniforms};
 
     for (long long round = 0; round < 2LL * N + 2; ++round) {
         bool any = false;
         for (int b = 0; b < B; ++b) any |= h_a[b] <= N;
         if (!any) break;
-        round_setup_kernel<<<(B + 127) / 128, 128, 0, s>>>(ra);
-        FREE_TRY(free_check_launch());
-        // (1) target step on the current state of every sample
-        PassIO io{};
-        io.x_in = w.x_cur; io.x_stride = d; io.t_idx = w.t_step; io.labels = labels;
-        io.mean_out = w.m_a; io.mean_stride = d; io.feat_out = K > 0 ? w.feat0 : nullptr;
-        FREE_TRY(target_pass(c, w, B, cfg, sch, io, s));
-        target_sample_kernel<<<egrid, 256, 0, s>>>(B, K, d, N, w.cur_a, w.active, w.t_step, sch->sigma2, w.m_a,
-                                                    noise_target, w.x_cur, w.pack_in);
-        FREE_TRY(free_check_launch());
-        if (K > 0) {
-            // (2) K drafter steps, each from the previous draft and feature
-            void* f_prev = w.feat0; void* f_next = w.feat1;
-            for (int i = 0; i < K; ++i) {
-                PassIO di{};
-                di.x_in = w.pack_in + (size_t)i * d; di.x_stride = (long long)K * d;         // x_hat_{a+i}
-                di.t_idx = w.t_draft + (size_t)i * B; di.labels = labels;
-                di.mean_out = w.m_draft + (size_t)i * d; di.mean_stride = (long long)K * d;
-                di.feat_out = f_next;
-                FREE_TRY(drafter_pass(c, w, B, cfg, sch, di, f_prev, s));
-                draft_sample_kernel<<<egrid, 256, 0, s>>>(B, K, d, N, i, w.cur_a, w.t_draft + (size_t)i * B, sch->sigma2,
-                                                           w.m_draft, noise_draft, w.x_draft, w.pack_in);
-                FREE_TRY(free_check_launch());
-                void* tmp = f_prev; f_prev = f_next; f_next = tmp;
-            }
-            // (3) one packed target pass over (x_a, x_hat_{a+1..a+K-1}) -> m_{a+1..a+K}
-            PassIO pi{};
-            pi.x_in = w.pack_in; pi.x_stride = d; pi.t_idx = w.t_pack; pi.labels = w.lab_pack;
-            pi.mean_out = w.m_target; pi.mean_stride = d;
-            FREE_TRY(target_pass(c, w, B * K, cfg, sch, pi, s));
-            // (4) sequential verification with the first-rejection break; the finalised state replaces x_cur
-            FREE_TRY(spec_verify(B, K, d, w.m_target, w.m_draft, w.x_draft, w.sigma2_bk, w.lam_bk, w.u_bk, w.nv,
-                                 w.x_cur, w.n_acc, nullptr, s));
-        }
-        cursor_update_kernel<<<(B + 127) / 128, 128, 0, s>>>(B, w.active, w.nv, w.n_acc, w.cur_a);
-        FREE_TRY(free_check_launch());
+        FREE_TRY(one_round(c, w, r, s));
         // host side of the round: cursors (loop control) and statistics
         FREE_CUDA_TRY(cudaMemcpyAsync(h_act.data(), w.active, B * 4, cudaMemcpyDeviceToHost, s));
         FREE_CUDA_TRY(cudaMemcpyAsync(h_nv.data(), w.nv, B * 4, cudaMemcpyDeviceToHost, s));
         if (K > 0) FREE_CUDA_TRY(cudaMemcpyAsync(h_acc.data(), w.n_acc, B * 4, cudaMemcpyDeviceToHost, s));
         FREE_CUDA_TRY(cudaMemcpyAsync(h_a.data(), w.cur_a, B * 4, cudaMemcpyDeviceToHost, s));
+        uint32_t dev_err = 0;
+        FREE_CUDA_TRY(cudaMemcpyAsync(&dev_err, w.err, 4, cudaMemcpyDeviceToHost, s));
         FREE_CUDA_TRY(cudaStreamSynchronize(s));
+        if (dev_err) return FREE_ERR_DEVICE_TIMEOUT;
         for (int b = 0; b < B; ++b) {
             if (!h_act[b]) continue;
             if (K > 0 && h_nv[b] > 0 && h_acc[b] < 0) return h_acc[b];
@@ -505,4 +600,38 @@ extern "C" int sample_trajectory(free_ctx* c, int B, const float* x0, const int3
     FREE_CUDA_TRY(cudaStreamSynchronize(s));
     if (stats && stats->target_calls > 0) stats->parallel_efficiency = (double)B * N / (double)stats->target_calls;
     return FREE_OK;
+}
+
+// ------------------------------------------------------------------------------------------------ profiling
+extern "C" int free_profile_begin(free_ctx* c) {
+    if (!c) return FREE_ERR_ARG;
+    for (ProfRec& r : c->prof) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
+    c->prof.clear();
+    c->prof_on = true;
+    return FREE_OK;
+}
+
+extern "C" int free_profile_end(free_ctx* c, free_prof_entry* out, int max_entries, int* n_entries) {
+    if (!c || !out || !n_entries || max_entries < 1) return FREE_ERR_ARG;
+    c->prof_on = false;
+    double ms[PC_N] = {}, work[PC_N] = {};
+    long long cnt[PC_N] = {};
+    int rc = FREE_OK;
+    for (ProfRec& r : c->prof) {
+        float t = 0.f;
+        if (cudaEventSynchronize(r.e1) != cudaSuccess || cudaEventElapsedTime(&t, r.e0, r.e1) != cudaSuccess) { (void)cudaGetLastError(); rc = FREE_ERR_CUDA; }
+        ms[r.cls] += t; work[r.cls] += r.work; cnt[r.cls] += 1;
+        cudaEventDestroy(r.e0); cudaEventDestroy(r.e1);
+    }
+    c->prof.clear();
+    int n = 0;
+    for (int k = 0; k < PC_N && n < max_entries; ++k) {
+        if (!cnt[k]) continue;
+        strncpy(out[n].name, kProfNames[k], sizeof(out[n].name) - 1);
+        out[n].name[sizeof(out[n].name) - 1] = 0;
+        out[n].launches = cnt[k]; out[n].ms = ms[k]; out[n].work = work[k];
+        ++n;
+    }
+    *n_entries = n;
+    return rc;
 }

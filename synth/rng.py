@@ -36,10 +36,15 @@ def round_to_bf16(a: np.ndarray) -> np.ndarray:
     numbers.
     """
     a = np.ascontiguousarray(a, dtype=np.float32)
-    bits = a.view(np.uint32).astype(np.uint64)
-    lsb = (bits >> np.uint64(16)) & np.uint64(1)
-    bits = (bits + np.uint64(0x7FFF) + lsb) & np.uint64(0xFFFF0000)
-    return bits.astype(np.uint32).view(np.float32).reshape(a.shape)
+    out = np.empty_like(a)
+    src, dst = a.reshape(-1).view(np.uint32), out.reshape(-1).view(np.uint32)
+    step = 1 << 24                                   # bounded temporaries for multi-GB tensors
+    for i in range(0, src.size, step):
+        bits = src[i:i + step]
+        lsb = (bits >> np.uint32(16)) & np.uint32(1)
+        # no finite input of interest is within 0x7fff of overflow, so uint32 arithmetic is exact here
+        dst[i:i + step] = (bits + (np.uint32(0x7FFF) + lsb)) & np.uint32(0xFFFF0000)
+    return out
 
 
 def to_bf16_bits(a: np.ndarray) -> np.ndarray:
