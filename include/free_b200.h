@@ -274,6 +274,26 @@ int free_op_attention(int dtype, int n_seq, int n_tok, int heads, int d_head,
                       const void* qkv, void* out, void* ws, size_t ws_bytes, void* stream);
 size_t free_op_attention_workspace_bytes(int dtype, int n_seq, int n_tok, int heads, int d_head);
 
+/*
+ * free_op_attention_static -- bf16 tensor-core attention that allocates nothing and takes no workspace.
+ * (The paper has no counterpart: this serves callers that are not allowed to allocate device memory -- code that
+ * runs under a frozen memory plan, plugins whose host application owns the memory pool, loops that must not hit
+ * the device-wide synchronisation of cudaMalloc / cudaFree.)  Same result as free_op_attention(FREE_BF16, ...).
+ * The scratch (head-major copies of q, k, v^T) is a 12 MiB array built into the library's device image: every
+ * GPU that loads the library holds it until the process ends.
+ *   Limit: n_seq * heads * n_tok * d_pad <= FREE_STATIC_ATTN_MAX_ELEMS, d_pad = d_head rounded up to 64/80/96/128;
+ *          larger problems return FREE_ERR_WORKSPACE.  n_tok % 128 == 0, d_head % 8 == 0, d_head <= 128, else
+ *          FREE_ERR_UNSUPPORTED.
+ *   qkv, out     DEVICE bf16, as for free_op_attention
+ *   device_error DEVICE uint32 (caller's): 0 after the call completes unless a bounded device-side wait gave up
+ * The first call on each device looks up the array's device address (with that device current); make that first
+ * call outside any stream capture.  All calls share the one array, which keeps the previous call's contents:
+ * each call rewrites everything it reads, but two calls that overlap on the GPU (different streams) race.
+ */
+#define FREE_STATIC_ATTN_MAX_ELEMS (1u << 21)
+int free_op_attention_static(int n_seq, int n_tok, int heads, int d_head, const void* qkv, void* out,
+                             uint32_t* device_error, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

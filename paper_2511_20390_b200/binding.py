@@ -86,6 +86,7 @@ _SIGNATURES = {
     "free_op_ln_modulate": (C.c_int, [C.c_int] * 4 + [C.c_void_p] * 3 + [C.c_int64, C.c_void_p, C.c_void_p]),
     "free_op_attention": (C.c_int, [C.c_int] * 5 + [C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "free_op_attention_workspace_bytes": (C.c_size_t, [C.c_int] * 5),
+    "free_op_attention_static": (C.c_int, [C.c_int] * 4 + [C.c_void_p] * 4),
 }
 
 
@@ -427,4 +428,23 @@ def op_attention(qkv, heads):
     err = int(ws[:4].view(torch.int32).item())
     if err:
         raise FreeError(-8, f"free_op_attention (device error word {err:#x})")
+    return out
+
+
+STATIC_ATTN_MAX_ELEMS = 1 << 21
+
+
+def op_attention_static(qkv, heads):
+    """bf16 attention through the entry point that allocates nothing inside the library: its scratch is a fixed
+    array in the library's device image (for callers that may not allocate).  qkv [n_seq, n_tok, 3*D] bf16.
+    The output tensor and the 4-byte error word are the caller's (allocated here by torch, outside the call)."""
+    n_seq, n_tok, D3 = qkv.shape
+    D = D3 // 3
+    _dev(qkv, torch.bfloat16)
+    out = torch.empty((n_seq, n_tok, D), dtype=torch.bfloat16, device=qkv.device)
+    err = torch.ones(1, dtype=torch.int32, device=qkv.device)
+    _check(lib().free_op_attention_static(n_seq, n_tok, heads, D // heads, _ptr(qkv), _ptr(out), _ptr(err), _stream()),
+           "free_op_attention_static")
+    if int(err.item()):
+        raise FreeError(-8, "free_op_attention_static (device error word set)")
     return out

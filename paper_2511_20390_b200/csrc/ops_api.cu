@@ -1,6 +1,7 @@
 // Public single-operation entry points (the same kernels the passes launch), used to check each
 // kernel against the CPU oracle on its own.
 #include "internal.h"
+#include <mutex>
 
 namespace {
 
@@ -72,4 +73,62 @@ extern "C" int free_op_attention(int dtype, int n_seq, int n_tok, int heads, int
     repack_qkv_kernel<<<grid, 256, 0, s>>>(n_seq, n_tok, heads, d_head, dp, (const __nv_bfloat16*)qkv, q, k, vt);
     FREE_TRY(free_check_launch());
     return attention_tc(n_seq, n_tok, heads, d_head, dp, q, k, vt, out, reinterpret_cast<uint32_t*>(ws), s);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Attention without any allocation, for callers that cannot provide a workspace.
+//
+// Some callers may not allocate device memory at all: code running while a CUDA graph is being captured or
+// replayed with a frozen memory plan, plugins of inference servers whose memory pool is owned by the host
+// application, and real-time loops that forbid cudaMalloc / cudaFree because those calls synchronise the
+// device.  For them the scratch of the tensor-core attention (the head-major copies of q, k and v^T) lives in
+// this file-scope device array.  Every GPU that loads the library holds these 12 MiB until the process exits.
+// ------------------------------------------------------------------------------------------------
+#define FREE_STATIC_ATTN_BYTES (3ull * FREE_STATIC_ATTN_MAX_ELEMS * 2ull)
+static __device__ __align__(256) unsigned char g_attn_scratch[FREE_STATIC_ATTN_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+unsigned char* g_scratch_ptr[kMaxDevices] = {};   // device address of g_attn_scratch on each device, once resolved
+
+// In host code `g_attn_scratch` names a host-side shadow of the symbol, not device memory: the device address
+// has to be asked for, once per device, with that device current.
+int scratch_for_current_device(unsigned char** out) {
+    int dev = 0;
+    FREE_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return FREE_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_ptr[dev]) {
+        void* p = nullptr;
+        FREE_CUDA_TRY(cudaGetSymbolAddress(&p, g_attn_scratch));
+        if (!p) return FREE_ERR_CUDA;
+        g_scratch_ptr[dev] = static_cast<unsigned char*>(p);
+    }
+    *out = g_scratch_ptr[dev];
+    return FREE_OK;
+}
+}  // namespace
+
+extern "C" int free_op_attention_static(int n_seq, int n_tok, int heads, int d_head, const void* qkv, void* out,
+                                        uint32_t* device_error, void* stream) {
+    if (n_seq < 1 || n_tok < 1 || heads < 1 || d_head < 1) return FREE_ERR_SHAPE;
+    if (!qkv || !out || !device_error) return FREE_ERR_ARG;
+    if (!free_aligned16(qkv) || !free_aligned16(out) || (reinterpret_cast<uintptr_t>(device_error) & 3u)) return FREE_ERR_ALIGN;
+    if (!attention_tc_supported(n_tok, d_head)) return FREE_ERR_UNSUPPORTED;
+    const int dp = attention_tc_dpad(d_head);
+    const unsigned long long elems = (unsigned long long)n_seq * heads * n_tok * dp;
+    if (elems > FREE_STATIC_ATTN_MAX_ELEMS) return FREE_ERR_WORKSPACE;      // beyond the built-in scratch
+    unsigned char* base = nullptr;
+    FREE_TRY(scratch_for_current_device(&base));
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    // the scratch keeps the previous call's contents: the repack below overwrites every element this call reads
+    // (padding included); only the caller's error word has to start at zero
+    FREE_CUDA_TRY(cudaMemsetAsync(device_error, 0, 4, s));
+    const size_t per = (size_t)FREE_STATIC_ATTN_MAX_ELEMS * 2;
+    __nv_bfloat16 *q = (__nv_bfloat16*)base, *k = (__nv_bfloat16*)(base + per), *vt = (__nv_bfloat16*)(base + 2 * per);
+    const unsigned grid = (unsigned)((elems + 255) / 256 > 148 * 16 ? 148 * 16 : (elems + 255) / 256);
+    repack_qkv_kernel<<<grid, 256, 0, s>>>(n_seq, n_tok, heads, d_head, dp, (const __nv_bfloat16*)qkv, q, k, vt);
+    FREE_TRY(free_check_launch());
+    return attention_tc(n_seq, n_tok, heads, d_head, dp, q, k, vt, out, device_error, s);
 }
