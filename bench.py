@@ -156,6 +156,9 @@ def make_workload(name, batch, rank):
         except ImportError:
             return VerifierWorkload(batch, rank)
         return RoundWorkload(batch, rank)
+    if name == "ops":
+        from bench_round import OpsWorkload
+        return OpsWorkload(batch, rank)
     raise SystemExit(f"unknown workload {name}")
 
 

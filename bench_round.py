@@ -160,3 +160,57 @@ def reference_arm(args, cores):
     return {"metric": RoundWorkload.metric, "value": val, "unit": "TFLOP/s", "ms_per_step": dt * 1e3, "dtype": "f64",
             "config": {"workload": "FREE round, DiT-XL/2-shaped 512^2, K=6, cfg 4, batch 16 (oracle: bounded sample)"},
             "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample}}
+
+
+class OpsWorkload:
+    """The hot kernels of one DiT-XL/2 block on their own, at 24 sequences of 1024 tokens (M = 24576 rows):
+    LayerNorm+modulate, QKV GEMM (head-major scatter is exercised by the full pass; here plain bias), attention,
+    proj GEMM (+gate, residual), fc1 GEMM (+GELU), fc2 GEMM (+gate, residual).  Used for profiling single kernels
+    on a case small enough for a full counter capture (inputs still exceed L2)."""
+    metric, unit, dtype = "DiT-XL/2 block kernels TFLOP/s", "TFLOP/s", "bf16"
+
+    def __init__(self, batch, rank):
+        import torch
+        from paper_2511_20390_b200 import binding as b
+        self.torch, self.b = torch, b
+        S, T, D, h = (batch or 24), 1024, 1152, 16
+        self.S, self.T, self.D, self.h = S, T, D, h
+        M, F = S * T, 4 * D
+        g = torch.Generator(device="cuda"); g.manual_seed(5 + rank)
+        rn = lambda *s, std=1.0: torch.randn(*s, generator=g, device="cuda") * std
+        self.x = rn(M, D)
+        self.mod = rn(S, 6 * D, std=0.1)
+        self.hn = rn(M, D).bfloat16()
+        self.qkv = rn(S, T, 3 * D).bfloat16()
+        self.hm = rn(M, F).bfloat16()
+        self.w = {k: rn(*s, std=0.02).bfloat16() for k, s in (("qkv", (3 * D, D)), ("proj", (D, D)), ("fc1", (F, D)), ("fc2", (D, F)))}
+        self.bias = {k: rn(v.shape[0], std=0.02) for k, v in self.w.items()}
+        self.flops = 2.0 * M * D * (3 * D + D + 2 * F) + 4.0 * S * h * T * T * (D // h)
+        self.units_per_step = self.flops / 1e12
+        self.launches_per_step = 6
+        self.config = {"workload": f"one DiT-XL/2 block's kernels, {S} sequences x 1024 tokens", "cache": "operands exceed L2"}
+
+    def step(self):
+        b = self.b
+        D = self.D
+        b.op_ln_modulate(self.x, self.mod[:, :D], self.mod[:, D:2 * D], self.T, out_dtype=b.FREE_BF16)
+        b.op_linear(self.hn, self.w["qkv"], self.bias["qkv"])
+        att = b.op_attention(self.qkv, self.h)
+        b.op_linear(att.view(-1, D), self.w["proj"], self.bias["proj"], epilogue=b.EPI_GATE_RESIDUAL, resid=self.x,
+                    gate=self.mod[:, 2 * D:3 * D], rows_per_seq=self.T)
+        b.op_linear(self.hn, self.w["fc1"], self.bias["fc1"], epilogue=b.EPI_BIAS_GELU)
+        b.op_linear(self.hm, self.w["fc2"], self.bias["fc2"], epilogue=b.EPI_GATE_RESIDUAL, resid=self.x,
+                    gate=self.mod[:, 5 * D:6 * D], rows_per_seq=self.T)
+
+    def host_step(self):
+        self.step()
+        return 0, 0
+
+    def roofline(self, ms, peaks):
+        ach = self.flops / 1e12 / (ms / 1e3)
+        return {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
+                "traffic": None, "kernel": "block kernels (aggregate)", "peak_source": peaks["source"]}
+
+    def oracle_sample(self):
+        import synth
+        return oracle_dit_sample(synth.DIT_XL2_512, 1)
