@@ -300,11 +300,31 @@ int launch(const CUtensorMap& mA, const CUtensorMap& mW, const TcArgs& a, size_t
 
 bool linear_bf16_supported(int N, int K) { return N >= 32 && N % 32 == 0 && K >= 64 && K % 64 == 0; }
 
+// Per-epilogue argument checks shared by the single-CTA and the CTA-pair kernels.
+static int validate_epilogue(const LinearArgs& l, long long ldo) {
+    switch (l.epi) {
+        case EPI_BIAS: case EPI_BIAS_GELU: case EPI_BIAS_SILU:
+            return (!l.out || !free_aligned16(l.out) || ldo % 8) ? FREE_ERR_ARG : FREE_OK;
+        case EPI_BIAS_EMB_SILU:
+            return (!l.out || !l.emb || !l.emb_idx || !free_aligned16(l.out) || ldo % 8) ? FREE_ERR_ARG : FREE_OK;
+        case EPI_GATE_RESIDUAL:
+            return (!l.resid || !free_aligned16(l.resid)) ? FREE_ERR_ARG : FREE_OK;
+        case EPI_QKV_HEADS:
+            return (!l.q || !l.k || !l.vt || l.heads < 1 || l.d_head % 8 || l.d_pad % 8 || l.d_pad < l.d_head || l.n_tok < 1 ||
+                    l.N != 3 * l.heads * l.d_head || l.M % l.n_tok) ? FREE_ERR_ARG : FREE_OK;
+        default:
+            return FREE_ERR_ARG;
+    }
+}
+
 int linear_bf16(const LinearArgs& l, cudaStream_t s) {
     if (l.M < 1 || !l.A || !l.W || !l.err) return FREE_ERR_ARG;
     if (!linear_bf16_supported(l.N, l.K)) return FREE_ERR_UNSUPPORTED;
     const long long lda = l.lda ? l.lda : l.K, ldw = l.ldw ? l.ldw : l.K, ldo = l.ldo ? l.ldo : l.N;
     if (lda % 8 || ldw % 8 || !free_aligned16(l.A) || !free_aligned16(l.W)) return FREE_ERR_ALIGN;
+    if (l.bias && !free_aligned16(l.bias)) return FREE_ERR_ALIGN;
+    FREE_TRY(validate_epilogue(l, ldo));
+    if (linear_bf16_pair_eligible(l)) return linear_bf16_pair(l, s);       // the large GEMMs: 256 x BN tiles on CTA pairs
     TcArgs a{};
     a.M = l.M; a.N = l.N; a.K = l.K;
     a.BN = pick_bn(l.N);
@@ -320,7 +340,6 @@ int linear_bf16(const LinearArgs& l, cudaStream_t s) {
     a.heads = l.heads; a.d_head = l.d_head; a.d_pad = l.d_pad; a.n_tok = l.n_tok;
     a.q = (__nv_bfloat16*)l.q; a.k = (__nv_bfloat16*)l.k; a.vt = (__nv_bfloat16*)l.vt;
     a.err = l.err;
-    if (l.bias && !free_aligned16(l.bias)) return FREE_ERR_ALIGN;
     const size_t smem = 1024 + kCtrlBytes + (size_t)a.stages * stage_bytes;
 
     CUtensorMap mA, mW;
@@ -330,23 +349,16 @@ int linear_bf16(const LinearArgs& l, cudaStream_t s) {
     const bool ob = l.out_dtype == FREE_BF16;
     switch (l.epi) {
         case EPI_BIAS:
-            if (!l.out || !free_aligned16(l.out) || ldo % 8) return FREE_ERR_ARG;
             return ob ? launch<EPI_BIAS, true>(mA, mW, a, smem, s) : launch<EPI_BIAS, false>(mA, mW, a, smem, s);
         case EPI_BIAS_GELU:
-            if (!l.out || !free_aligned16(l.out) || ldo % 8) return FREE_ERR_ARG;
             return ob ? launch<EPI_BIAS_GELU, true>(mA, mW, a, smem, s) : launch<EPI_BIAS_GELU, false>(mA, mW, a, smem, s);
         case EPI_BIAS_SILU:
-            if (!l.out || !free_aligned16(l.out) || ldo % 8) return FREE_ERR_ARG;
             return ob ? launch<EPI_BIAS_SILU, true>(mA, mW, a, smem, s) : launch<EPI_BIAS_SILU, false>(mA, mW, a, smem, s);
         case EPI_BIAS_EMB_SILU:
-            if (!l.out || !l.emb || !l.emb_idx || !free_aligned16(l.out) || ldo % 8) return FREE_ERR_ARG;
             return ob ? launch<EPI_BIAS_EMB_SILU, true>(mA, mW, a, smem, s) : launch<EPI_BIAS_EMB_SILU, false>(mA, mW, a, smem, s);
         case EPI_GATE_RESIDUAL:
-            if (!l.resid || !free_aligned16(l.resid)) return FREE_ERR_ARG;
             return launch<EPI_GATE_RESIDUAL, false>(mA, mW, a, smem, s);
         case EPI_QKV_HEADS:
-            if (!l.q || !l.k || !l.vt || l.heads < 1 || l.d_head % 8 || l.d_pad % 8 || l.d_pad < l.d_head || l.n_tok < 1 ||
-                l.N != 3 * l.heads * l.d_head || l.M % l.n_tok) return FREE_ERR_ARG;
             return launch<EPI_QKV_HEADS, true>(mA, mW, a, smem, s);
         default:
             return FREE_ERR_ARG;

@@ -1,0 +1,361 @@
+// bf16 linear layers on CTA pairs (tcgen05 cta_group::2): the kernel behind the large GEMMs of the DiT blocks.
+//
+//   out = epilogue(A[M,K] * W[N,K]^T + bias),   A and W bf16 (K contiguous), fp32 accumulation in TMEM.
+//
+// Why pairs: a 128 x 256 tile per SM needs 48 KB of operands per 64-wide K step, and the L2 -> SM path
+// (about 48 B per clock per SM) then holds the tensor core to half rate.  Two CTAs of a cluster that share
+// one 256 x BN tile each load their own 128 rows of A and only HALF of the W rows (32 KB per K step); the
+// MMA reads both halves across the pair.  No multicast loads are used anywhere.
+//
+// Persistent kernel, one CTA per SM, clusters of two, 192 threads per CTA:
+//   warp 0     TMA producer (both CTAs): its A rows and its W half into a ring of stages; completion is
+//              counted on the even CTA's mbarrier, which expects the bytes of both CTAs;
+//   warp 1     MMA issuer (even CTA only): tcgen05.mma.cta_group::2, 256 x BN x 16 per instruction, two TMEM
+//              accumulators per CTA; stage-release and accumulator-ready barriers are signalled in both CTAs;
+//   warps 2-5  epilogue (both CTAs, each on its own 128 rows): tcgen05.ld, fused bias / GELU / gate, then
+//              through swizzled shared-memory staging to a TMA store, or a TMA add-reduction for the gated
+//              residual update (the fp32 residual stream is never read by the SM).  The QKV variant scatters
+//              straight into the head-major attention operands.
+// Tile order: N fastest, so the clusters in flight share a few row blocks of A while W stays in L2.
+#include "internal.h"
+#include "tc_common.cuh"
+#include <mutex>
+
+namespace {
+
+constexpr int BK = 64;
+constexpr int kThreads = 192;
+constexpr int kMaxStages = 8;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kABytes = 128 * BK * 2;              // one CTA's A tile of a stage
+constexpr uint32_t kCtrlBytes = 1024;
+constexpr uint32_t kStageBufBytes = 4096;               // 32 rows x 128 bytes
+constexpr uint32_t kStagingBytes = 4 * 2 * kStageBufBytes;
+constexpr uint32_t kSmemBudget = 227 * 1024;
+
+struct Tc2Args {
+    int M, N, K, num_m, num_n, stages;
+    const float* bias;
+    const float* gate; long long gate_stride; int rows_per_seq;
+    int heads, d_head, d_pad, n_tok;
+    __nv_bfloat16 *q, *k, *vt;
+    uint32_t* err;
+};
+
+__device__ __forceinline__ float tanh_fast(float x) { float y; asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+__device__ __forceinline__ float gelu_fast(float a) {
+    return 0.5f * a * (1.0f + tanh_fast(0.7978845608028654f * (a + 0.044715f * a * a * a)));
+}
+__device__ __forceinline__ uint4 pack8(const float* v) {
+    __nv_bfloat162 p0 = __floats2bfloat162_rn(v[0], v[1]), p1 = __floats2bfloat162_rn(v[2], v[3]);
+    __nv_bfloat162 p2 = __floats2bfloat162_rn(v[4], v[5]), p3 = __floats2bfloat162_rn(v[6], v[7]);
+    uint4 u;
+    u.x = *reinterpret_cast<uint32_t*>(&p0); u.y = *reinterpret_cast<uint32_t*>(&p1);
+    u.z = *reinterpret_cast<uint32_t*>(&p2); u.w = *reinterpret_cast<uint32_t*>(&p3);
+    return u;
+}
+
+// Head-major scatter of one row's 32 columns [n0, n0+32) of the QKV output (d_head % 8 == 0).
+__device__ __forceinline__ void scatter_qkv(const Tc2Args& a, int row, int n0, const float* v) {
+    const int D = a.heads * a.d_head, dh = a.d_head, dp = a.d_pad, T = a.n_tok;
+    const int seq = row / T, tok = row % T;
+    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        const int n = n0 + 8 * g;
+        const int which = n / D, hd = (n % D) / dh, c = n % dh;
+        const long long sh = (long long)seq * a.heads + hd;
+        if (which < 2) {
+            __nv_bfloat16* dst = (which == 0 ? a.q : a.k) + (sh * T + tok) * dp + c;
+            *reinterpret_cast<uint4*>(dst) = pack8(v + 8 * g);
+            if (c + 8 == dh)
+                for (int z = dh; z < dp; z += 8) *reinterpret_cast<uint4*>(dst + (z - c)) = zero;
+        } else {
+            __nv_bfloat16* dst = a.vt + (sh * dp + c) * T + tok;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) dst[(long long)i * T] = __float2bfloat16(v[8 * g + i]);
+            if (c + 8 == dh)
+                for (int z = dh; z < dp; ++z) a.vt[(sh * dp + z) * T + tok] = __float2bfloat16(0.f);
+        }
+    }
+}
+
+template <int EPI, bool OUT_BF16, int BN>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapW,
+                  const __grid_constant__ CUtensorMap mapO, const Tc2Args a) {
+    constexpr uint32_t kBBytes = (BN / 2) * BK * 2;          // one CTA's half of the W tile of a stage
+    constexpr uint32_t kStageBytes = kABytes + kBBytes;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem);      // used in the even CTA only
+    uint64_t* empty = full + kMaxStages;
+    uint64_t* accf = empty + kMaxStages;
+    uint64_t* acce = accf + 2;                               // used in the even CTA only
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acce + 2);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+    uint8_t* staging = smem + kCtrlBytes;
+    uint8_t* tiles = staging + kStagingBytes;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = tc::cluster_ctarank();
+    const int stages = a.stages, nk = a.K / BK;
+    const long long total = (long long)a.num_m * a.num_n;
+    const long long first = tc::cluster_id_x(), step = tc::num_clusters_x();
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
+        for (int i = 0; i < 2; ++i) { tc::mbar_init(&accf[i], 1); tc::mbar_init(&acce[i], 8); }
+        *abort_flag = 0;
+        tc::fence_barrier_init();
+        tc::fence_proxy_async();
+    }
+    if (warp == 1) { tc::tmem_alloc_pair(tmem_slot, kTmemCols); tc::tmem_relinquish_pair(); }
+    tc::tc_fence_before();
+    tc::cluster_sync_all();                                  // barriers of both CTAs initialised before any remote use
+    tc::tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    auto fail = [&](uint32_t code) { *abort_flag = 1; atomicOr(a.err, code); };
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (both CTAs)
+        if (lane == 0) {
+            tc::tma_prefetch_desc(&mapA);
+            tc::tma_prefetch_desc(&mapW);
+            const uint32_t full0 = tc::mapa(tc::smem_u32(&full[0]), 0);      // the even CTA's stage barriers
+            uint32_t it = 0;
+            bool ok = true;
+            for (long long t = first; ok && t < total; t += step) {
+                const int m_blk = (int)(t / a.num_n), n_blk = (int)(t % a.num_n);
+                const int a_row = m_blk * 256 + (int)rank * 128, w_row = n_blk * BN + (int)rank * (BN / 2);
+                for (int kb = 0; kb < nk; ++kb, ++it) {
+                    const int s = it % stages;
+                    const uint32_t ph = (it / stages) & 1u;
+                    if (*abort_flag || !tc::mbar_wait(&empty[s], ph ^ 1u)) { fail(FREE_DEV_ERR_EMPTY_WAIT); ok = false; break; }
+                    const uint32_t dst = tc::smem_u32(tiles + (size_t)s * kStageBytes);
+                    if (rank == 0) tc::mbar_expect_tx(&full[s], 2 * kStageBytes);
+                    tc::tma_load_2d_pair(dst, &mapA, full0 + 8u * s, kb * BK, a_row);
+                    tc::tma_load_2d_pair(dst + kABytes, &mapW, full0 + 8u * s, kb * BK, w_row);
+                }
+            }
+            if (!ok || *abort_flag) {
+                // loads in flight must land before the shared memory is given back: they take microseconds
+                const uint64_t t0 = tc::global_ns();
+                while (tc::global_ns() - t0 < 200000ull) { }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (even CTA only)
+        if (rank == 0 && lane == 0) {
+            const uint32_t idesc = tc::idesc_bf16(256, BN);
+            uint32_t it = 0, tl = 0;
+            bool ok = true;
+            for (long long t = first; ok && t < total; t += step, ++tl) {
+                const uint32_t acc = tl & 1u, aph = (tl >> 1) & 1u;
+                if (*abort_flag || !tc::mbar_wait(&acce[acc], aph ^ 1u)) { fail(FREE_DEV_ERR_ACC_EMPTY); ok = false; break; }
+                tc::tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * (uint32_t)BN;
+                for (int kb = 0; kb < nk; ++kb, ++it) {
+                    const int s = it % stages;
+                    const uint32_t ph = (it / stages) & 1u;
+                    if (*abort_flag || !tc::mbar_wait(&full[s], ph)) { fail(FREE_DEV_ERR_FULL_WAIT); ok = false; break; }
+                    tc::tc_fence_after();
+                    const uint32_t a_addr = tc::smem_u32(tiles + (size_t)s * kStageBytes), b_addr = a_addr + kABytes;
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)
+                        tc::mma_bf16_pair(d_tmem, tc::smem_desc(a_addr + k * 32, 1024, 2), tc::smem_desc(b_addr + k * 32, 1024, 2),
+                                          idesc, (kb | k) != 0 ? 1u : 0u);
+                    tc::mma_commit_pair(&empty[s]);          // both CTAs may refill the stage once these MMAs have read it
+                }
+                if (ok) tc::mma_commit_pair(&accf[acc]);     // accumulators complete in both CTAs
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ epilogue (both CTAs)
+        const int q = warp & 3;                              // TMEM lanes [32q, 32q+32) belong to this warp
+        const uint32_t acce0 = tc::mapa(tc::smem_u32(&acce[0]), 0);
+        uint8_t* my_stage = staging + (size_t)q * 2 * kStageBufBytes;
+        constexpr int CH = OUT_BF16 ? 64 : 32;               // columns per staging buffer (128 bytes per row)
+        uint32_t tl = 0, nst = 0;
+        for (long long t = first; t < total; t += step, ++tl) {
+            const int m_blk = (int)(t / a.num_n), n_blk = (int)(t % a.num_n);
+            const uint32_t acc = tl & 1u, aph = (tl >> 1) & 1u;
+            const bool bad = *abort_flag || !tc::mbar_wait(&accf[acc], aph);
+            if (__any_sync(0xffffffffu, bad)) { if (lane == 0) fail(FREE_DEV_ERR_ACC_FULL); break; }
+            tc::tc_fence_after();
+            const int row0 = m_blk * 256 + (int)rank * 128 + q * 32;
+            const int row = row0 + lane;
+            const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * (uint32_t)BN;
+            if (EPI == EPI_QKV_HEADS) {
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    uint32_t r[32];
+                    tc::tmem_ld32(t_addr + (uint32_t)c0, r);
+                    tc::tmem_wait_ld();
+                    if (row < a.M) {
+                        const int n0 = n_blk * BN + c0;
+                        float v[32];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const float4 b = __ldg(reinterpret_cast<const float4*>(a.bias + n0) + i);
+                            v[4 * i + 0] = __uint_as_float(r[4 * i + 0]) + b.x; v[4 * i + 1] = __uint_as_float(r[4 * i + 1]) + b.y;
+                            v[4 * i + 2] = __uint_as_float(r[4 * i + 2]) + b.z; v[4 * i + 3] = __uint_as_float(r[4 * i + 3]) + b.w;
+                        }
+                        scatter_qkv(a, row, n0, v);
+                    }
+                }
+            } else {
+                const int rowc = row < a.M ? row : a.M - 1;
+                const float* gp = (EPI == EPI_GATE_RESIDUAL && a.gate) ? a.gate + (long long)(rowc / a.rows_per_seq) * a.gate_stride : nullptr;
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN; c0 += CH) {
+                    const int n0 = n_blk * BN + c0;
+                    float v[CH];
+#pragma unroll
+                    for (int h = 0; h < CH / 32; ++h) {
+                        uint32_t r[32];
+                        tc::tmem_ld32(t_addr + (uint32_t)(c0 + 32 * h), r);
+                        tc::tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[32 * h + i] = __uint_as_float(r[i]);
+                    }
+                    if (a.bias) {
+#pragma unroll
+                        for (int i = 0; i < CH / 4; ++i) {
+                            const float4 b = __ldg(reinterpret_cast<const float4*>(a.bias + n0) + i);
+                            v[4 * i + 0] += b.x; v[4 * i + 1] += b.y; v[4 * i + 2] += b.z; v[4 * i + 3] += b.w;
+                        }
+                    }
+                    if (EPI == EPI_BIAS_GELU) {
+#pragma unroll
+                        for (int i = 0; i < CH; ++i) v[i] = gelu_fast(v[i]);
+                    }
+                    if (EPI == EPI_GATE_RESIDUAL && gp) {
+                        const bool gvec = (reinterpret_cast<uintptr_t>(gp + n0) & 15u) == 0;
+#pragma unroll
+                        for (int i = 0; i < CH / 4; ++i) {
+                            float4 g;
+                            if (gvec) g = __ldg(reinterpret_cast<const float4*>(gp + n0) + i);
+                            else g = make_float4(__ldg(gp + n0 + 4 * i), __ldg(gp + n0 + 4 * i + 1), __ldg(gp + n0 + 4 * i + 2), __ldg(gp + n0 + 4 * i + 3));
+                            v[4 * i + 0] *= g.x; v[4 * i + 1] *= g.y; v[4 * i + 2] *= g.z; v[4 * i + 3] *= g.w;
+                        }
+                    }
+                    // stage the 32 x 128-byte block (16-byte units XOR-swizzled by row, as the tensor map expects)
+                    uint8_t* buf = my_stage + (nst & 1u) * kStageBufBytes;
+                    if (lane == 0) tc::bulk_wait_read<1>();              // the store issued from this buffer two chunks ago has read it
+                    __syncwarp();
+                    uint8_t* rowp = buf + lane * 128;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        uint4 w;
+                        if (OUT_BF16) w = pack8(v + 8 * u);
+                        else w = make_uint4(__float_as_uint(v[4 * u]), __float_as_uint(v[4 * u + 1]), __float_as_uint(v[4 * u + 2]), __float_as_uint(v[4 * u + 3]));
+                        *reinterpret_cast<uint4*>(rowp + ((u ^ (lane & 7)) << 4)) = w;
+                    }
+                    tc::fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (row0 < a.M) {                                // rows past M inside the box are clipped by the TMA unit
+                            if (EPI == EPI_GATE_RESIDUAL) tc::tma_reduce_add_2d(&mapO, tc::smem_u32(buf), n0, row0);
+                            else tc::tma_store_2d(&mapO, tc::smem_u32(buf), n0, row0);
+                        }
+                        tc::bulk_commit();
+                    }
+                    ++nst;
+                }
+            }
+            tc::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive_cluster(acce0 + 8u * acc);
+        }
+        if (lane == 0) tc::bulk_wait<0>();                   // every store of this warp complete before the CTA ends
+        __syncwarp();
+    }
+    // ---------------------------------------------------------------------- teardown
+    tc::tc_fence_before();
+    tc::cluster_sync_all();                                  // the peer may still read this CTA's shared memory until here
+    if (warp == 1) { tc::tc_fence_after(); tc::tmem_dealloc_pair(tmem_base, kTmemCols); }
+}
+
+int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 2) n = 148;
+    }
+    return n;
+}
+
+template <int EPI, bool OUT_BF16, int BN>
+int launch(const CUtensorMap& mA, const CUtensorMap& mW, const CUtensorMap& mO, const Tc2Args& a, size_t smem, cudaStream_t s) {
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [&] {
+        attr_err = cudaFuncSetAttribute(linear_tc2_kernel<EPI, OUT_BF16, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget);
+    });
+    if (attr_err != cudaSuccess) return FREE_ERR_CUDA;
+    const long long tiles = (long long)a.num_m * a.num_n;
+    const long long pairs = sm_count() / 2;
+    const int grid = 2 * (int)(tiles < pairs ? tiles : pairs);
+    linear_tc2_kernel<EPI, OUT_BF16, BN><<<grid, kThreads, smem, s>>>(mA, mW, mO, a);
+    return free_check_launch();
+}
+
+template <int BN>
+int dispatch(const LinearArgs& l, Tc2Args a, cudaStream_t s) {
+    constexpr uint32_t stage_bytes = kABytes + (BN / 2) * BK * 2;
+    a.stages = (int)((kSmemBudget - 1024 - kCtrlBytes - kStagingBytes) / stage_bytes);
+    if (a.stages > kMaxStages) a.stages = kMaxStages;
+    a.num_m = (l.M + 255) / 256; a.num_n = l.N / BN;
+    const size_t smem = 1024 + kCtrlBytes + kStagingBytes + (size_t)a.stages * stage_bytes;
+    const long long lda = l.lda ? l.lda : l.K, ldw = l.ldw ? l.ldw : l.K, ldo = l.ldo ? l.ldo : l.N;
+    CUtensorMap mA, mW, mO;
+    FREE_TRY(free_tensor_map_2d(&mA, l.A, (uint64_t)l.K, (uint64_t)l.M, (uint64_t)lda * 2, BK, 128, 128));
+    FREE_TRY(free_tensor_map_2d(&mW, l.W, (uint64_t)l.K, (uint64_t)l.N, (uint64_t)ldw * 2, BK, BN / 2, 128));
+    const bool ob = l.out_dtype == FREE_BF16;
+    switch (l.epi) {
+        case EPI_BIAS:
+            FREE_TRY(free_tensor_map_2d_typed(&mO, ob ? 2 : 4, l.out, (uint64_t)l.N, (uint64_t)l.M, (uint64_t)ldo * (ob ? 2 : 4), ob ? 64 : 32, 32, 128));
+            return ob ? launch<EPI_BIAS, true, BN>(mA, mW, mO, a, smem, s) : launch<EPI_BIAS, false, BN>(mA, mW, mO, a, smem, s);
+        case EPI_BIAS_GELU:
+            FREE_TRY(free_tensor_map_2d_typed(&mO, 2, l.out, (uint64_t)l.N, (uint64_t)l.M, (uint64_t)ldo * 2, 64, 32, 128));
+            return launch<EPI_BIAS_GELU, true, BN>(mA, mW, mO, a, smem, s);
+        case EPI_GATE_RESIDUAL:
+            FREE_TRY(free_tensor_map_2d_typed(&mO, 4, l.resid, (uint64_t)l.N, (uint64_t)l.M, (uint64_t)l.N * 4, 32, 32, 128));
+            return launch<EPI_GATE_RESIDUAL, false, BN>(mA, mW, mO, a, smem, s);
+        case EPI_QKV_HEADS:
+            mO = mA;                                         // unused by this variant
+            return launch<EPI_QKV_HEADS, true, BN>(mA, mW, mO, a, smem, s);
+        default:
+            return FREE_ERR_UNSUPPORTED;
+    }
+}
+
+}  // namespace
+
+// Shapes and epilogues the pair kernel takes; everything else stays on the single-CTA kernel.
+bool linear_bf16_pair_eligible(const LinearArgs& l) {
+    if (l.M <= 128 || l.K < BK || l.K % BK) return false;
+    if (l.N % 256 && l.N % 192) return false;
+    switch (l.epi) {
+        case EPI_BIAS: return l.out != nullptr;
+        case EPI_BIAS_GELU: return l.out != nullptr && l.out_dtype == FREE_BF16;
+        case EPI_GATE_RESIDUAL: return l.resid != nullptr;
+        case EPI_QKV_HEADS: return l.bias != nullptr;
+        default: return false;
+    }
+}
+
+// Arguments have been validated by linear_bf16().
+int linear_bf16_pair(const LinearArgs& l, cudaStream_t s) {
+    Tc2Args a{};
+    a.M = l.M; a.N = l.N; a.K = l.K;
+    a.bias = l.bias;
+    a.gate = l.gate; a.gate_stride = l.gate_stride; a.rows_per_seq = l.rows_per_seq > 0 ? l.rows_per_seq : 1;
+    a.heads = l.heads; a.d_head = l.d_head; a.d_pad = l.d_pad; a.n_tok = l.n_tok;
+    a.q = (__nv_bfloat16*)l.q; a.k = (__nv_bfloat16*)l.k; a.vt = (__nv_bfloat16*)l.vt;
+    a.err = l.err;
+    return l.N % 256 == 0 ? dispatch<256>(l, a, s) : dispatch<192>(l, a, s);
+}

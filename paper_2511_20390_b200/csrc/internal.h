@@ -33,6 +33,8 @@ struct LinearArgs {
 int linear_fp32(const LinearArgs& a, cudaStream_t s);   // CUDA cores, any sizes
 int linear_bf16(const LinearArgs& a, cudaStream_t s);   // tcgen05; K % 64 == 0, N % 16 == 0
 bool linear_bf16_supported(int N, int K);
+bool linear_bf16_pair_eligible(const LinearArgs& a);    // large shapes run on CTA pairs (256 x BN tiles)
+int linear_bf16_pair(const LinearArgs& a, cudaStream_t s);
 
 // ---- attention -------------------------------------------------------------------------------
 // token-major qkv [n_seq, n_tok, 3, heads, d_head] -> out [n_seq, n_tok, heads*d_head]

@@ -30,14 +30,21 @@ CUtensorMapSwizzle swz(int bytes) {
 
 int free_tensor_map_2d(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t outer_stride_bytes,
                        uint32_t box_inner, uint32_t box_outer, int swizzle_bytes) {
+    return free_tensor_map_2d_typed(map, 2, base, inner, outer, outer_stride_bytes, box_inner, box_outer, swizzle_bytes);
+}
+
+int free_tensor_map_2d_typed(CUtensorMap* map, int elem_bytes, const void* base, uint64_t inner, uint64_t outer,
+                             uint64_t outer_stride_bytes, uint32_t box_inner, uint32_t box_outer, int swizzle_bytes) {
     auto fn = encode_fn();
     if (!fn) return FREE_ERR_CUDA;
-    if (box_inner * 2u > (uint32_t)swizzle_bytes || box_outer > 256 || outer_stride_bytes % 16) return FREE_ERR_UNSUPPORTED;
+    if (elem_bytes != 2 && elem_bytes != 4) return FREE_ERR_ARG;
+    if (box_inner * (uint32_t)elem_bytes > (uint32_t)swizzle_bytes || box_outer > 256 || outer_stride_bytes % 16) return FREE_ERR_UNSUPPORTED;
     cuuint64_t dims[2] = {inner, outer};
     cuuint64_t strides[1] = {outer_stride_bytes};
     cuuint32_t box[2] = {box_inner, box_outer};
     cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+    CUresult r = fn(map, elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                    const_cast<void*>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, swz(swizzle_bytes), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? FREE_OK : FREE_ERR_CUDA;

@@ -18,7 +18,8 @@ def _operands(M, N, K, seed):
 
 
 SHAPES = [(128, 32, 64), (128, 256, 64), (256, 192, 128), (300, 384, 192), (96, 64, 256), (1, 128, 64),
-          (1000, 1152, 1152), (777, 3456, 384), (40000, 384, 64), (19500, 160, 128), (640, 4608, 1152), (512, 1152, 4608)]
+          (1000, 1152, 1152), (777, 3456, 384), (40000, 384, 64), (19500, 160, 128), (640, 4608, 1152), (512, 1152, 4608),
+          (9000, 3456, 384), (6100, 4608, 128), (129, 192, 64)]
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES)
@@ -39,6 +40,7 @@ def test_epilogues(M, N, K):
     a_, w_, b_ = cu(A, torch.bfloat16), cu(W, torch.bfloat16), cu(bias)
     assert nerr(b.op_linear(a_, w_, b_), ref) < 5e-3                                        # bf16 output rounding
     assert nerr(b.op_linear(a_, w_, b_, epilogue=b.EPI_BIAS_GELU, out_dtype=b.FREE_FP32), odit.gelu_tanh(ref)) < 1.5e-3   # tanh.approx
+    assert nerr(b.op_linear(a_, w_, b_, epilogue=b.EPI_BIAS_GELU), odit.gelu_tanh(ref)) < 5e-3             # bf16 output
     assert nerr(b.op_linear(a_, w_, b_, epilogue=b.EPI_BIAS_SILU, out_dtype=b.FREE_FP32), odit.silu(ref)) < 1e-5
     assert nerr(b.op_linear(a_, w_, None, out_dtype=b.FREE_FP32), ref - bias) < 1e-5
     rps = 64
