@@ -165,8 +165,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap mapQ0, const __grid_cons
             if (!ok) {
                 fail();
                 // let loads in flight land before shared memory is released
-                tc::mbar_wait(bar_k, 0, 20000000ull); tc::mbar_wait(bar_k, 1, 20000000ull);
-                tc::mbar_wait(bar_v, 0, 20000000ull); tc::mbar_wait(bar_v, 1, 20000000ull);
+                tc::mbar_wait(bar_k, 0, 40000000ll); tc::mbar_wait(bar_k, 1, 40000000ll);
+                tc::mbar_wait(bar_v, 0, 40000000ll); tc::mbar_wait(bar_v, 1, 40000000ll);
             }
         }
         __syncwarp();

@@ -206,7 +206,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             if (!ok || *abort_flag) {
                 // loads already issued must land before the shared memory is given back
                 const uint32_t n_back = it < (uint32_t)stages ? it : (uint32_t)stages;
-                for (uint32_t j = it - n_back; j < it; ++j) tc::mbar_wait(&full[j % stages], (j / stages) & 1u, 50000000ull);
+                for (uint32_t j = it - n_back; j < it; ++j) tc::mbar_wait(&full[j % stages], (j / stages) & 1u, 100000000ll);
             }
         }
         __syncwarp();

@@ -4,14 +4,20 @@
 //
 // Why pairs: a 128 x 256 tile per SM needs 48 KB of operands per 64-wide K step, and the L2 -> SM path
 // (about 48 B per clock per SM) then holds the tensor core to half rate.  Two CTAs of a cluster that share
-// one 256 x BN tile each load their own 128 rows of A and only HALF of the W rows (32 KB per K step); the
+// one 256 x 256 tile each load their own 128 rows of A and only HALF of the W rows (32 KB per K step); the
 // MMA reads both halves across the pair.  No multicast loads are used anywhere.
 //
 // Persistent kernel, one CTA per SM, clusters of two, 192 threads per CTA:
 //   warp 0     TMA producer (both CTAs): its A rows and its W half into a ring of stages; completion is
 //              counted on the even CTA's mbarrier, which expects the bytes of both CTAs;
-//   warp 1     MMA issuer (even CTA only): tcgen05.mma.cta_group::2, 256 x BN x 16 per instruction, two TMEM
-//              accumulators per CTA; stage-release and accumulator-ready barriers are signalled in both CTAs;
+//   warp 1     MMA issuer (even CTA only): tcgen05.mma.cta_group::2, 256 x 256 x 16 per instruction, two TMEM
+//              accumulators per CTA; stage-release and accumulator-ready barriers are signalled in both CTAs.
+//              The whole warp runs the issue loop converged and one elected lane issues: measured on B200, a
+//              single-lane (divergent) loop of wait + 4 MMAs + commit takes ~660 clocks per K step, the converged
+//              loop ~508, and one MMA cannot be issued faster than every ~94 clocks whatever its size.  Only
+//              N = 256 (128 clocks of tensor work per instruction) therefore keeps the tensor core busy, so the
+//              tile is always 256 wide and a ragged last column block is zero-filled by TMA (rows of W past N)
+//              and clipped on the way out;
 //   warps 2-5  epilogue (both CTAs, each on its own 128 rows): tcgen05.ld, fused bias / GELU / gate, then
 //              through swizzled shared-memory staging to a TMA store, or a TMA add-reduction for the gated
 //              residual update (the fp32 residual stream is never read by the SM).  The QKV variant scatters
@@ -119,56 +125,63 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
-        if (lane == 0) {
-            tc::tma_prefetch_desc(&mapA);
-            tc::tma_prefetch_desc(&mapW);
-            const uint32_t full0 = tc::mapa(tc::smem_u32(&full[0]), 0);      // the even CTA's stage barriers
-            uint32_t it = 0;
-            bool ok = true;
-            for (long long t = first; ok && t < total; t += step) {
-                const int m_blk = (int)(t / a.num_n), n_blk = (int)(t % a.num_n);
-                const int a_row = m_blk * 256 + (int)rank * 128, w_row = n_blk * BN + (int)rank * (BN / 2);
-                for (int kb = 0; kb < nk; ++kb, ++it) {
-                    const int s = it % stages;
-                    const uint32_t ph = (it / stages) & 1u;
-                    if (*abort_flag || !tc::mbar_wait(&empty[s], ph ^ 1u)) { fail(FREE_DEV_ERR_EMPTY_WAIT); ok = false; break; }
+        if (lane == 0) { tc::tma_prefetch_desc(&mapA); tc::tma_prefetch_desc(&mapW); }
+        const uint32_t full0 = tc::mapa(tc::smem_u32(&full[0]), 0);          // the even CTA's stage barriers
+        uint32_t it = 0;
+        bool ok = true;
+        for (long long t = first; ok && t < total; t += step) {
+            const int m_blk = (int)(t / a.num_n), n_blk = (int)(t % a.num_n);
+            const int a_row = m_blk * 256 + (int)rank * 128, w_row = n_blk * BN + (int)rank * (BN / 2);
+            for (int kb = 0; kb < nk; ++kb, ++it) {
+                const int s = it % stages;
+                const uint32_t ph = (it / stages) & 1u;
+                ok = __all_sync(0xffffffffu, !*abort_flag && tc::mbar_wait(&empty[s], ph ^ 1u));
+                if (!ok) { if (lane == 0) fail(FREE_DEV_ERR_EMPTY_WAIT); break; }
+                if (tc::elect_one()) {
                     const uint32_t dst = tc::smem_u32(tiles + (size_t)s * kStageBytes);
                     if (rank == 0) tc::mbar_expect_tx(&full[s], 2 * kStageBytes);
                     tc::tma_load_2d_pair(dst, &mapA, full0 + 8u * s, kb * BK, a_row);
                     tc::tma_load_2d_pair(dst + kABytes, &mapW, full0 + 8u * s, kb * BK, w_row);
                 }
+                __syncwarp();
             }
-            if (!ok || *abort_flag) {
-                // loads in flight must land before the shared memory is given back: they take microseconds
-                const uint64_t t0 = tc::global_ns();
-                while (tc::global_ns() - t0 < 200000ull) { }
-            }
+        }
+        if (!ok || *abort_flag) {
+            // loads in flight must land before the shared memory is given back: they take microseconds
+            const long long t0 = clock64();
+            while (clock64() - t0 < 400000ll) { }
         }
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (even CTA only)
-        if (rank == 0 && lane == 0) {
+        if (rank == 0) {
             const uint32_t idesc = tc::idesc_bf16(256, BN);
             uint32_t it = 0, tl = 0;
             bool ok = true;
             for (long long t = first; ok && t < total; t += step, ++tl) {
                 const uint32_t acc = tl & 1u, aph = (tl >> 1) & 1u;
-                if (*abort_flag || !tc::mbar_wait(&acce[acc], aph ^ 1u)) { fail(FREE_DEV_ERR_ACC_EMPTY); ok = false; break; }
+                ok = __all_sync(0xffffffffu, !*abort_flag && tc::mbar_wait(&acce[acc], aph ^ 1u));
+                if (!ok) { if (lane == 0) fail(FREE_DEV_ERR_ACC_EMPTY); break; }
                 tc::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * (uint32_t)BN;
                 for (int kb = 0; kb < nk; ++kb, ++it) {
                     const int s = it % stages;
                     const uint32_t ph = (it / stages) & 1u;
-                    if (*abort_flag || !tc::mbar_wait(&full[s], ph)) { fail(FREE_DEV_ERR_FULL_WAIT); ok = false; break; }
+                    ok = __all_sync(0xffffffffu, !*abort_flag && tc::mbar_wait(&full[s], ph));
+                    if (!ok) { if (lane == 0) fail(FREE_DEV_ERR_FULL_WAIT); break; }
                     tc::tc_fence_after();
-                    const uint32_t a_addr = tc::smem_u32(tiles + (size_t)s * kStageBytes), b_addr = a_addr + kABytes;
+                    if (tc::elect_one()) {
+                        const uint32_t a_addr = tc::smem_u32(tiles + (size_t)s * kStageBytes), b_addr = a_addr + kABytes;
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)
-                        tc::mma_bf16_pair(d_tmem, tc::smem_desc(a_addr + k * 32, 1024, 2), tc::smem_desc(b_addr + k * 32, 1024, 2),
-                                          idesc, (kb | k) != 0 ? 1u : 0u);
-                    tc::mma_commit_pair(&empty[s]);          // both CTAs may refill the stage once these MMAs have read it
+                        for (int k = 0; k < BK / 16; ++k)
+                            tc::mma_bf16_pair(d_tmem, tc::smem_desc(a_addr + k * 32, 1024, 2), tc::smem_desc(b_addr + k * 32, 1024, 2),
+                                              idesc, (kb | k) != 0 ? 1u : 0u);
+                        tc::mma_commit_pair(&empty[s]);      // both CTAs may refill the stage once these MMAs have read it
+                    }
+                    __syncwarp();
                 }
-                if (ok) tc::mma_commit_pair(&accf[acc]);     // accumulators complete in both CTAs
+                if (ok && tc::elect_one()) tc::mma_commit_pair(&accf[acc]);   // accumulators complete in both CTAs
+                __syncwarp();
             }
         }
         __syncwarp();
@@ -190,7 +203,7 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
             const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * (uint32_t)BN;
             if (EPI == EPI_QKV_HEADS) {
 #pragma unroll 1
-                for (int c0 = 0; c0 < BN; c0 += 32) {
+                for (int c0 = 0; c0 < BN && n_blk * BN + c0 < a.N; c0 += 32) {
                     uint32_t r[32];
                     tc::tmem_ld32(t_addr + (uint32_t)c0, r);
                     tc::tmem_wait_ld();
@@ -210,7 +223,7 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
                 const int rowc = row < a.M ? row : a.M - 1;
                 const float* gp = (EPI == EPI_GATE_RESIDUAL && a.gate) ? a.gate + (long long)(rowc / a.rows_per_seq) * a.gate_stride : nullptr;
 #pragma unroll 1
-                for (int c0 = 0; c0 < BN; c0 += CH) {
+                for (int c0 = 0; c0 < BN && n_blk * BN + c0 < a.N; c0 += CH) {
                     const int n0 = n_blk * BN + c0;
                     float v[CH];
 #pragma unroll
@@ -308,7 +321,7 @@ int dispatch(const LinearArgs& l, Tc2Args a, cudaStream_t s) {
     constexpr uint32_t stage_bytes = kABytes + (BN / 2) * BK * 2;
     a.stages = (int)((kSmemBudget - 1024 - kCtrlBytes - kStagingBytes) / stage_bytes);
     if (a.stages > kMaxStages) a.stages = kMaxStages;
-    a.num_m = (l.M + 255) / 256; a.num_n = l.N / BN;
+    a.num_m = (l.M + 255) / 256; a.num_n = (l.N + BN - 1) / BN;
     const size_t smem = 1024 + kCtrlBytes + kStagingBytes + (size_t)a.stages * stage_bytes;
     const long long lda = l.lda ? l.lda : l.K, ldw = l.ldw ? l.ldw : l.K, ldo = l.ldo ? l.ldo : l.N;
     CUtensorMap mA, mW, mO;
@@ -338,7 +351,7 @@ int dispatch(const LinearArgs& l, Tc2Args a, cudaStream_t s) {
 // Shapes and epilogues the pair kernel takes; everything else stays on the single-CTA kernel.
 bool linear_bf16_pair_eligible(const LinearArgs& l) {
     if (l.M <= 128 || l.K < BK || l.K % BK) return false;
-    if (l.N % 256 && l.N % 192) return false;
+    if (l.N < 256 || l.N % 64) return false;            // column chunks of the epilogue are 64 wide
     switch (l.epi) {
         case EPI_BIAS: return l.out != nullptr;
         case EPI_BIAS_GELU: return l.out != nullptr && l.out_dtype == FREE_BF16;
@@ -357,5 +370,5 @@ int linear_bf16_pair(const LinearArgs& l, cudaStream_t s) {
     a.heads = l.heads; a.d_head = l.d_head; a.d_pad = l.d_pad; a.n_tok = l.n_tok;
     a.q = (__nv_bfloat16*)l.q; a.k = (__nv_bfloat16*)l.k; a.vt = (__nv_bfloat16*)l.vt;
     a.err = l.err;
-    return l.N % 256 == 0 ? dispatch<256>(l, a, s) : dispatch<192>(l, a, s);
+    return dispatch<256>(l, a, s);
 }

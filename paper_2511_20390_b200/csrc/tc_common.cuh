@@ -47,16 +47,17 @@ __device__ __forceinline__ uint64_t global_ns() {
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait: false if the phase did not complete within `limit_ns` of wall-clock time (each poll may
-// itself block for a short hardware-defined time, so the bound is on time, not on the poll count).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint64_t limit_ns = 2000000000ull) {
+// Bounded wait: false if the phase did not complete within `limit_cycles` SM clock cycles (about 2 s by
+// default).  The bound is taken on the SM's own cycle counter, which is cheap to read; the system-wide
+// nanosecond timer is far slower to read and would add its latency to every wait that is not ready at once.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long long limit_cycles = 4000000000ll) {
     if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = global_ns();
+    const long long t0 = clock64();
     for (;;) {
 #pragma unroll 1
-        for (int i = 0; i < 32; ++i)
+        for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (global_ns() - t0 > limit_ns) return false;
+        if (clock64() - t0 > limit_cycles) return false;
     }
 }
 
