@@ -37,25 +37,72 @@ __global__ void cond_setup_kernel(int n_states, int G, int freq_dim, int n_class
 
 // ---------------------------------------------------------------------------------------------
 // Patch embedding: token (i, j) of a state gathers its C*p*p patch (order: channel, row, column),
-// out = pe_w . patch + pe_b + pos[token].  One CTA per (state, token); written once per guidance stream.
+// out = pe_w . patch + pe_b + pos[token], written once per guidance stream.  Thread t of a CTA owns output
+// channels t, t + 256, ... and keeps their weight rows in registers (PD = C p p values each); the CTA walks
+// over (state, token) pairs, so weights are read once per CTA and every store is a coalesced row segment.
+template <typename T, int PD, int CPT>
+__global__ void __launch_bounds__(256) patch_embed_kernel(int n_items, int G, int C, int H, int W, int p, int D,
+                                                          const float* __restrict__ x_in, long long x_stride,
+                                                          const float* __restrict__ pe_w, const float* __restrict__ pe_b,
+                                                          const float* __restrict__ pos, T* __restrict__ out) {
+    __shared__ float patch[2][PD];
+    const int gw = W / p, n_tok = (H / p) * gw;
+    float w[CPT][PD], b[CPT];
+#pragma unroll
+    for (int j = 0; j < CPT; ++j) {
+        const int o = threadIdx.x + j * 256;
+        b[j] = o < D ? pe_b[o] : 0.f;
+#pragma unroll
+        for (int e = 0; e < PD; ++e) w[j][e] = o < D ? pe_w[(long long)o * PD + e] : 0.f;
+    }
+    auto gather = [&](int item, float* dst) {
+        if (threadIdx.x < PD && item < n_items) {
+            const int st = item / n_tok, tok = item % n_tok, ti = tok / gw, tj = tok % gw;
+            const int e = threadIdx.x, c = e / (p * p), r = (e / p) % p, cc = e % p;
+            dst[e] = x_in[(long long)st * x_stride + ((long long)c * H + ti * p + r) * W + tj * p + cc];
+        }
+    };
+    int item = blockIdx.x, buf = 0;
+    gather(item, patch[0]);
+    __syncthreads();
+    for (; item < n_items; item += gridDim.x, buf ^= 1) {
+        gather(item + gridDim.x, patch[buf ^ 1]);                 // next item's patch while this one is used
+        const int st = item / n_tok, tok = item % n_tok;
+#pragma unroll
+        for (int j = 0; j < CPT; ++j) {
+            const int o = threadIdx.x + j * 256;
+            if (o < D) {
+                float acc = 0.f;
+#pragma unroll
+                for (int e = 0; e < PD; ++e) acc = fmaf(w[j][e], patch[buf][e], acc);
+                acc += b[j] + __ldg(pos + (long long)tok * D + o);
+                for (int g = 0; g < G; ++g)
+                    store_act(out + ((long long)(st * G + g) * n_tok + tok) * D + o, acc);
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// Any patch size / width: one CTA per (state, token), weights read from global memory.
 template <typename T>
-__global__ void __launch_bounds__(128) patch_embed_kernel(int G, int C, int H, int W, int p, int D,
-                                                          const float* x_in, long long x_stride, const float* pe_w,
-                                                          const float* pe_b, const float* pos, T* out) {
-    extern __shared__ float patch[];
+__global__ void __launch_bounds__(128) patch_embed_generic_kernel(int G, int C, int H, int W, int p, int D,
+                                                                  const float* x_in, long long x_stride, const float* pe_w,
+                                                                  const float* pe_b, const float* pos, T* out) {
+    extern __shared__ float patch_dyn[];
     const int gw = W / p, n_tok = (H / p) * gw, pd = C * p * p;
     const int st = blockIdx.x / n_tok, tok = blockIdx.x % n_tok;
     const int ti = tok / gw, tj = tok % gw;
     const float* x = x_in + (long long)st * x_stride;
     for (int e = threadIdx.x; e < pd; e += blockDim.x) {
         int c = e / (p * p), r = (e / p) % p, cc = e % p;
-        patch[e] = x[((long long)c * H + ti * p + r) * W + tj * p + cc];
+        patch_dyn[e] = x[((long long)c * H + ti * p + r) * W + tj * p + cc];
     }
     __syncthreads();
     for (int o = threadIdx.x; o < D; o += blockDim.x) {
         const float* w = pe_w + (long long)o * pd;
         float acc = 0.f;
-        for (int e = 0; e < pd; ++e) acc = fmaf(w[e], patch[e], acc);
+        for (int e = 0; e < pd; ++e) acc = fmaf(w[e], patch_dyn[e], acc);
         acc += pe_b[o] + pos[(long long)tok * D + o];
         for (int g = 0; g < G; ++g)
             store_act(out + ((long long)(st * G + g) * n_tok + tok) * D + o, acc);
@@ -64,67 +111,99 @@ __global__ void __launch_bounds__(128) patch_embed_kernel(int G, int C, int H, i
 
 // ---------------------------------------------------------------------------------------------
 // LayerNorm (no affine, eps 1e-6, biased variance, two-pass statistics) + y = ln (1 + scale) + shift.
-// One warp per row.  VPL > 0: the row (D = 128 * VPL) lives in registers as VPL float4 per lane.
+// One warp per row.  VPL > 0: the row (D = 128 * VPL) lives in registers as VPL float4 per lane; warps stride
+// over the rows and issue the loads of their next row before reducing the current one, so that each warp always
+// has a full row of 16-byte loads in flight (the kernel is a pure stream: read 4 D, write 2 D or 4 D bytes per row).
 template <typename T, int VPL>
-__global__ void __launch_bounds__(256) ln_modulate_kernel(int M, int D, int rows_per_seq, const float* x,
-                                                          const float* shift, const float* scale, long long mod_stride, T* y) {
-    const int row = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
+__global__ void __launch_bounds__(256, 2) ln_modulate_kernel(int M, int D, int rows_per_seq, const float* __restrict__ x,
+                                                             const float* __restrict__ shift, const float* __restrict__ scale,
+                                                             long long mod_stride, T* __restrict__ y) {
     const int lane = threadIdx.x % 32;
-    if (row >= M) return;
-    const float* xr = x + (long long)row * D;
-    const long long mo = (long long)(row / rows_per_seq) * mod_stride;
+    const int warps = gridDim.x * (blockDim.x / 32);
+    int row = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
     const float invD = 1.f / (float)D;
     if (VPL > 0) {
-        float4 v[VPL > 0 ? VPL : 1];
-        float s = 0.f;
+        float4 v[VPL > 0 ? VPL : 1], nx[VPL > 0 ? VPL : 1];
+        if (row < M) {
 #pragma unroll
-        for (int i = 0; i < VPL; ++i) {
-            v[i] = reinterpret_cast<const float4*>(xr)[i * 32 + lane];
-            s += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+            for (int i = 0; i < VPL; ++i) nx[i] = __ldcs(reinterpret_cast<const float4*>(x + (long long)row * D) + i * 32 + lane);
         }
-        const float mu = free_warp_sum(s) * invD;
-        float q = 0.f;
+        for (; row < M; row += warps) {
 #pragma unroll
-        for (int i = 0; i < VPL; ++i) {
-            float a = v[i].x - mu, b = v[i].y - mu, c = v[i].z - mu, d = v[i].w - mu;
-            q += (a * a + b * b) + (c * c + d * d);
-        }
-        const float rstd = rsqrtf(free_warp_sum(q) * invD + 1e-6f);
+            for (int i = 0; i < VPL; ++i) v[i] = nx[i];
+            const int next = row + warps;
+            if (next < M) {
 #pragma unroll
-        for (int i = 0; i < VPL; ++i) {
-            const int c0 = (i * 32 + lane) * 4;
-            const float4 sh = *reinterpret_cast<const float4*>(shift + mo + c0);
-            const float4 sc = *reinterpret_cast<const float4*>(scale + mo + c0);
-            float o0 = (v[i].x - mu) * rstd * (1.f + sc.x) + sh.x;
-            float o1 = (v[i].y - mu) * rstd * (1.f + sc.y) + sh.y;
-            float o2 = (v[i].z - mu) * rstd * (1.f + sc.z) + sh.z;
-            float o3 = (v[i].w - mu) * rstd * (1.f + sc.w) + sh.w;
-            if (sizeof(T) == 4) {
-                reinterpret_cast<float4*>(y + (long long)row * D)[i * 32 + lane] = make_float4(o0, o1, o2, o3);
-            } else {
-                __nv_bfloat162 lo = __floats2bfloat162_rn(o0, o1), hi = __floats2bfloat162_rn(o2, o3);
-                uint2 pk;
-                pk.x = *reinterpret_cast<uint32_t*>(&lo);
-                pk.y = *reinterpret_cast<uint32_t*>(&hi);
-                reinterpret_cast<uint2*>(y + (long long)row * D)[i * 32 + lane] = pk;
+                for (int i = 0; i < VPL; ++i) nx[i] = __ldcs(reinterpret_cast<const float4*>(x + (long long)next * D) + i * 32 + lane);
+            }
+            const long long mo = (long long)(row / rows_per_seq) * mod_stride;
+            float s = 0.f;
+#pragma unroll
+            for (int i = 0; i < VPL; ++i) s += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+            const float mu = free_warp_sum(s) * invD;
+            float q = 0.f;
+#pragma unroll
+            for (int i = 0; i < VPL; ++i) {
+                float a = v[i].x - mu, b = v[i].y - mu, c = v[i].z - mu, d = v[i].w - mu;
+                q += (a * a + b * b) + (c * c + d * d);
+            }
+            const float rstd = rsqrtf(free_warp_sum(q) * invD + 1e-6f);
+#pragma unroll
+            for (int i = 0; i < VPL; ++i) {
+                const int c0 = (i * 32 + lane) * 4;
+                const float4 sh = __ldg(reinterpret_cast<const float4*>(shift + mo + c0));
+                const float4 sc = __ldg(reinterpret_cast<const float4*>(scale + mo + c0));
+                float o0 = (v[i].x - mu) * rstd * (1.f + sc.x) + sh.x;
+                float o1 = (v[i].y - mu) * rstd * (1.f + sc.y) + sh.y;
+                float o2 = (v[i].z - mu) * rstd * (1.f + sc.z) + sh.z;
+                float o3 = (v[i].w - mu) * rstd * (1.f + sc.w) + sh.w;
+                if (sizeof(T) == 4) {
+                    reinterpret_cast<float4*>(y + (long long)row * D)[i * 32 + lane] = make_float4(o0, o1, o2, o3);
+                } else {
+                    __nv_bfloat162 lo = __floats2bfloat162_rn(o0, o1), hi = __floats2bfloat162_rn(o2, o3);
+                    uint2 pk;
+                    pk.x = *reinterpret_cast<uint32_t*>(&lo);
+                    pk.y = *reinterpret_cast<uint32_t*>(&hi);
+                    reinterpret_cast<uint2*>(y + (long long)row * D)[i * 32 + lane] = pk;
+                }
             }
         }
     } else {
-        float s = 0.f;
-        for (int c = lane; c < D; c += 32) s += xr[c];
-        const float mu = free_warp_sum(s) * invD;
-        float q = 0.f;
-        for (int c = lane; c < D; c += 32) { float a = xr[c] - mu; q += a * a; }
-        const float rstd = rsqrtf(free_warp_sum(q) * invD + 1e-6f);
-        for (int c = lane; c < D; c += 32)
-            store_act(y + (long long)row * D + c, (xr[c] - mu) * rstd * (1.f + scale[mo + c]) + shift[mo + c]);
+        for (; row < M; row += warps) {
+            const float* xr = x + (long long)row * D;
+            const long long mo = (long long)(row / rows_per_seq) * mod_stride;
+            float s = 0.f;
+            for (int c = lane; c < D; c += 32) s += xr[c];
+            const float mu = free_warp_sum(s) * invD;
+            float q = 0.f;
+            for (int c = lane; c < D; c += 32) { float a = xr[c] - mu; q += a * a; }
+            const float rstd = rsqrtf(free_warp_sum(q) * invD + 1e-6f);
+            for (int c = lane; c < D; c += 32)
+                store_act(y + (long long)row * D + c, (xr[c] - mu) * rstd * (1.f + scale[mo + c]) + shift[mo + c]);
+        }
     }
 }
 
 template <typename T>
-__global__ void convert_kernel(long long n, const float* x, T* y) {
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
-        store_act(y + i, x[i]);
+__global__ void convert_kernel(long long n, const float* __restrict__ x, T* __restrict__ y) {
+    const long long n4 = n / 4, stride = (long long)gridDim.x * blockDim.x, i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y)) & 15u) == 0) {
+        for (long long i = i0; i < n4; i += stride) {
+            const float4 v = __ldcs(reinterpret_cast<const float4*>(x) + i);
+            if (sizeof(T) == 4) {
+                reinterpret_cast<float4*>(y)[i] = v;
+            } else {
+                __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+                uint2 pk;
+                pk.x = *reinterpret_cast<uint32_t*>(&lo);
+                pk.y = *reinterpret_cast<uint32_t*>(&hi);
+                reinterpret_cast<uint2*>(y)[i] = pk;
+            }
+        }
+        for (long long i = n4 * 4 + i0; i < n; i += stride) store_act(y + i, x[i]);
+    } else {
+        for (long long i = i0; i < n; i += stride) store_act(y + i, x[i]);
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -185,23 +264,40 @@ int cond_setup(int dtype, int n_states, int G, int freq_dim, int n_classes, int 
     return free_check_launch();
 }
 
+template <typename T>
+static int patch_embed_launch(int n_states, int G, int C, int H, int W, int p, int D, const float* x_in, long long x_stride,
+                              const float* pe_w, const float* pe_b, const float* pos, T* out, cudaStream_t s) {
+    const int n_tok = (H / p) * (W / p), pd = C * p * p;
+    const int n_items = n_states * n_tok;
+    if (pd == 16 && D <= 5 * 256) {                   // the DiT */2 models: 4 channels, 2 x 2 patches
+        const unsigned grid = (unsigned)(n_items < 148 * 4 ? n_items : 148 * 4);
+        const int cpt = (D + 255) / 256;
+        switch (cpt) {
+            case 1: patch_embed_kernel<T, 16, 1><<<grid, 256, 0, s>>>(n_items, G, C, H, W, p, D, x_in, x_stride, pe_w, pe_b, pos, out); break;
+            case 2: patch_embed_kernel<T, 16, 2><<<grid, 256, 0, s>>>(n_items, G, C, H, W, p, D, x_in, x_stride, pe_w, pe_b, pos, out); break;
+            case 3: patch_embed_kernel<T, 16, 3><<<grid, 256, 0, s>>>(n_items, G, C, H, W, p, D, x_in, x_stride, pe_w, pe_b, pos, out); break;
+            case 4: patch_embed_kernel<T, 16, 4><<<grid, 256, 0, s>>>(n_items, G, C, H, W, p, D, x_in, x_stride, pe_w, pe_b, pos, out); break;
+            default: patch_embed_kernel<T, 16, 5><<<grid, 256, 0, s>>>(n_items, G, C, H, W, p, D, x_in, x_stride, pe_w, pe_b, pos, out); break;
+        }
+    } else {
+        patch_embed_generic_kernel<T><<<(unsigned)n_items, 128, (size_t)pd * sizeof(float), s>>>(G, C, H, W, p, D, x_in, x_stride, pe_w, pe_b, pos, out);
+    }
+    return free_check_launch();
+}
+
 int patch_embed(int out_dtype, int n_states, int G, int C, int H, int W, int p, int D,
                 const float* x_in, long long x_stride, const float* pe_w, const float* pe_b, const float* pos,
                 void* out, cudaStream_t s) {
-    const int n_tok = (H / p) * (W / p);
-    const size_t smem = (size_t)C * p * p * sizeof(float);
-    const unsigned grid = (unsigned)(n_states * n_tok);
-    if (out_dtype == FREE_FP32)
-        patch_embed_kernel<float><<<grid, 128, smem, s>>>(G, C, H, W, p, D, x_in, x_stride, pe_w, pe_b, pos, (float*)out);
-    else
-        patch_embed_kernel<__nv_bfloat16><<<grid, 128, smem, s>>>(G, C, H, W, p, D, x_in, x_stride, pe_w, pe_b, pos, (__nv_bfloat16*)out);
-    return free_check_launch();
+    return out_dtype == FREE_FP32
+        ? patch_embed_launch<float>(n_states, G, C, H, W, p, D, x_in, x_stride, pe_w, pe_b, pos, (float*)out, s)
+        : patch_embed_launch<__nv_bfloat16>(n_states, G, C, H, W, p, D, x_in, x_stride, pe_w, pe_b, pos, (__nv_bfloat16*)out, s);
 }
 
 template <typename T>
 static int ln_launch(int M, int D, int rps, const float* x, const float* sh, const float* sc, long long ms, T* y, cudaStream_t s) {
-    const int rows_per_cta = 8;
-    const unsigned grid = (unsigned)((M + rows_per_cta - 1) / rows_per_cta);
+    const int rows_per_cta = 8;                       // one warp per row; persistent: 2 CTAs of 8 warps per SM
+    const unsigned need = (unsigned)((M + rows_per_cta - 1) / rows_per_cta), cap = 148u * 2u;
+    const unsigned grid = need < cap ? need : cap;
     const bool vec = (D % 128 == 0) && (ms % 4 == 0) && free_aligned16(sh) && free_aligned16(sc) && free_aligned16(x) && free_aligned16(y);
     const int vpl = vec ? D / 128 : 0;
     switch (vpl) {
