@@ -1,0 +1,394 @@
+// Non-causal multi-head self-attention on the 5th-generation tensor cores, two query tiles per CTA.
+//
+// One CTA (one per SM) owns 256 queries of one (sequence, head): two tiles of 128 queries that alternate on the
+// tensor core, so that the softmax of one tile runs while the MMAs of the other execute.
+//   warps 0-3   softmax + output accumulation of query tile 0 (thread = one query row = one TMEM lane)
+//   warps 4-7   the same for query tile 1
+//   warp 8      TMA producer: Q tiles once, then K and V^T blocks of 128 keys into double buffers
+//   warp 9      MMA issuer (the warp runs converged, one elected lane issues):
+//               S_t = Q_t K^T (128 x 128 x d_pad) into TMEM, O_t = P_t V (128 x d_pad x 128) into TMEM
+// Per block of 128 keys and per tile: wait S, fold the previous block's O into the fp32 register accumulator
+// (rescaled by the running-max correction), two passes over S in TMEM (row maximum; exp2, row sum, P rounded to
+// bf16 and stored to shared memory in the MMA operand layout), signal P.  The issue order
+// PV_0, S_0(next), PV_1, S_1(next) keeps one tile's MMAs in flight while the other tile is in its softmax.
+//
+// Operands.  q and k are read straight from a token-major bf16 matrix [n_seq * n_tok, ld] (the output of the QKV
+// linear layer): head h of q starts at column q_col0 + h * d_head, of k at k_col0 + h * d_head.  d_pad is 64 plus a
+// tail of 0 / 16 / 32 columns (its own 32- / 64-byte swizzle).  When d_head is not 64 + tail, the tail's last columns
+// belong to the next head: they are zeroed in the Q tiles after loading (the matching K columns then multiply
+// zeros).  v^T is head-major [n_seq * heads, d_pad, n_tok] (rows past d_head are never used: they only feed
+// output columns that are not stored).  Output: [n_seq * n_tok, heads * d_head] bf16.
+#include "internal.h"
+#include "tc_common.cuh"
+#include <mutex>
+
+namespace {
+
+constexpr int BQ = 128, BKV = 128;
+constexpr int kThreads = 320;
+constexpr uint32_t kTmemCols = 512;           // S_0 [0,128), S_1 [128,256), O_0 [256,384), O_1 [384,512)
+
+struct Attn2Args {
+    int n_tok, heads, d_head;
+    int q_col0, k_col0;
+    float scale_log2e;
+    __nv_bfloat16* out;
+    uint32_t* err;
+};
+
+template <int DP> struct Geo2 {
+    static constexpr int W1 = DP - 64;                                  // tail chunk: 0, 16 or 32 columns
+    static constexpr uint32_t LAY1 = W1 == 32 ? 4 : 6;                  // 64- or 32-byte swizzle
+    static constexpr uint32_t ROW1 = W1 * 2;                            // bytes per row of the tail chunk
+    static constexpr uint32_t QK0_BYTES = 128 * 128;
+    static constexpr uint32_t QK1_BYTES = 128 * ROW1;
+    static constexpr uint32_t QK_BYTES = QK0_BYTES + QK1_BYTES;         // one Q or K tile (multiple of 1024)
+    static constexpr uint32_t V_HALF = DP * 128;                        // DP rows x 64 keys
+    static constexpr uint32_t V_BYTES = 2 * V_HALF;
+    static constexpr uint32_t P_HALF = 128 * 128;
+    static constexpr uint32_t P_BYTES = 2 * P_HALF;
+    static constexpr uint32_t OFF_Q = 0;                                // two tiles
+    static constexpr uint32_t OFF_K = OFF_Q + 2 * QK_BYTES;             // two buffers
+    static constexpr uint32_t OFF_V = OFF_K + 2 * QK_BYTES;             // two buffers
+    static constexpr uint32_t OFF_P = OFF_V + 2 * V_BYTES;              // two tiles
+    static constexpr uint32_t TILE_BYTES = OFF_P + 2 * P_BYTES;
+    static constexpr uint32_t SMEM = 1024 /*align*/ + 1024 /*barriers*/ + TILE_BYTES;
+    static_assert(QK_BYTES % 1024 == 0 && V_HALF % 1024 == 0, "tiles must keep the swizzle alignment");
+    static_assert(SMEM <= 227 * 1024, "does not fit in shared memory");
+};
+
+__device__ __forceinline__ float ex2(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+
+template <int DP>
+__global__ void __launch_bounds__(kThreads, 1)
+attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_constant__ CUtensorMap mapQK1,
+                     const __grid_constant__ CUtensorMap mapV, const Attn2Args a) {
+    using G = Geo2<DP>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t* bar_q = reinterpret_cast<uint64_t*>(smem);
+    uint64_t* bar_qz = bar_q + 1;       // Q tiles fixed up (padding columns zeroed): one arrival per softmax warp
+    uint64_t* k_full = bar_q + 2;       // [2]
+    uint64_t* k_empty = bar_q + 4;      // [2]
+    uint64_t* v_full = bar_q + 6;       // [2]
+    uint64_t* v_empty = bar_q + 8;      // [2]
+    uint64_t* s_full = bar_q + 10;      // [2] per tile: S complete
+    uint64_t* p_ready = bar_q + 12;     // [2] per tile: P stored and S consumed (4 warp arrivals)
+    uint64_t* o_full = bar_q + 14;      // [2] per tile: O_j complete
+    uint64_t* o_free = bar_q + 16;      // [2] per tile: O_j folded into registers (4 warp arrivals)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_q + 18);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+    uint8_t* tiles = smem + 1024;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int sh = blockIdx.y;                              // sequence * heads + head
+    const int seq = sh / a.heads, head = sh % a.heads;
+    const int q0 = blockIdx.x * 2 * BQ;
+    const int T = a.n_tok, nb = T / BKV;
+    const int nq = (q0 + BQ < T) ? 2 : 1;                   // query tiles this CTA really has
+
+    if (threadIdx.x == 0) {
+        tc::mbar_init(bar_q, 1); tc::mbar_init(bar_qz, 4 * nq);
+        for (int i = 0; i < 2; ++i) {
+            tc::mbar_init(&k_full[i], 1); tc::mbar_init(&k_empty[i], 1); tc::mbar_init(&v_full[i], 1); tc::mbar_init(&v_empty[i], 1);
+            tc::mbar_init(&s_full[i], 1); tc::mbar_init(&p_ready[i], 4); tc::mbar_init(&o_full[i], 1); tc::mbar_init(&o_free[i], 4);
+        }
+        *abort_flag = 0;
+        tc::fence_barrier_init();
+        tc::fence_proxy_async();
+    }
+    if (warp == 9) { tc::tmem_alloc(tmem_slot, kTmemCols); tc::tmem_relinquish(); }
+    tc::tc_fence_before();
+    __syncthreads();
+    tc::tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    auto fail = [&]() { *abort_flag = 1; atomicOr(a.err, FREE_DEV_ERR_ATTN); };
+    // warp-uniform bounded wait; false = give up
+    auto wait = [&](uint64_t* bar, uint32_t parity) -> bool {
+        return __all_sync(0xffffffffu, !*abort_flag && tc::mbar_wait(bar, parity));
+    };
+
+    if (warp == 8) {
+        // ------------------------------------------------------------------ TMA producer
+        const int row_q = seq * T + q0;                     // row of the first query in the token-major matrix
+        const int xq = a.q_col0 + head * a.d_head, xk = a.k_col0 + head * a.d_head;
+        const int v_row = sh * DP;
+        if (lane == 0) { tc::tma_prefetch_desc(&mapQK0); tc::tma_prefetch_desc(&mapV); }
+        if (tc::elect_one()) {
+            tc::mbar_expect_tx(bar_q, (uint32_t)nq * G::QK_BYTES);
+            for (int t = 0; t < nq; ++t) {
+                uint8_t* sQ = tiles + G::OFF_Q + t * G::QK_BYTES;
+                tc::tma_load_2d(sQ, &mapQK0, bar_q, xq, row_q + t * BQ);
+                if (G::W1 > 0) tc::tma_load_2d(sQ + G::QK0_BYTES, &mapQK1, bar_q, xq + 64, row_q + t * BQ);
+            }
+        }
+        __syncwarp();
+        bool ok = true;
+        for (int j = 0; ok && j < nb; ++j) {
+            const int b = j & 1;
+            const uint32_t ph = (uint32_t)(j >> 1) & 1u;
+            ok = wait(&k_empty[b], ph ^ 1u);
+            if (!ok) break;
+            if (tc::elect_one()) {
+                uint8_t* sK = tiles + G::OFF_K + b * G::QK_BYTES;
+                tc::mbar_expect_tx(&k_full[b], G::QK_BYTES);
+                tc::tma_load_2d(sK, &mapQK0, &k_full[b], xk, seq * T + j * BKV);
+                if (G::W1 > 0) tc::tma_load_2d(sK + G::QK0_BYTES, &mapQK1, &k_full[b], xk + 64, seq * T + j * BKV);
+            }
+            __syncwarp();
+            ok = wait(&v_empty[b], ph ^ 1u);
+            if (!ok) break;
+            if (tc::elect_one()) {
+                uint8_t* sV = tiles + G::OFF_V + b * G::V_BYTES;
+                tc::mbar_expect_tx(&v_full[b], G::V_BYTES);
+                tc::tma_load_2d(sV, &mapV, &v_full[b], j * BKV, v_row);
+                tc::tma_load_2d(sV + G::V_HALF, &mapV, &v_full[b], j * BKV + 64, v_row);
+            }
+            __syncwarp();
+        }
+        if (!ok) {
+            if (lane == 0) fail();
+            const long long t0 = clock64();                 // loads in flight land within microseconds
+            while (clock64() - t0 < 400000ll) { }
+        }
+        __syncwarp();
+    } else if (warp == 9) {
+        // ------------------------------------------------------------------ MMA issuer
+        const uint32_t idesc_s = tc::idesc_bf16(BQ, BKV), idesc_o = tc::idesc_bf16(BQ, DP);
+        const uint32_t q_base = tc::smem_u32(tiles + G::OFF_Q), k_base = tc::smem_u32(tiles + G::OFF_K);
+        const uint32_t v_base = tc::smem_u32(tiles + G::OFF_V), p_base = tc::smem_u32(tiles + G::OFF_P);
+        auto issue_s = [&](int t, int kb) {                 // S_t = Q_t K^T over d_pad in steps of 16 (elected lane)
+            const uint32_t qa = q_base + t * G::QK_BYTES, ka = k_base + kb * G::QK_BYTES, d = tmem_base + t * 128;
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                tc::mma_bf16(d, tc::smem_desc(qa + k * 32, 1024, 2), tc::smem_desc(ka + k * 32, 1024, 2), idesc_s, k != 0);
+#pragma unroll
+            for (int k = 0; k < G::W1 / 16; ++k)
+                tc::mma_bf16(d, tc::smem_desc(qa + G::QK0_BYTES + k * 32, 8 * G::ROW1, G::LAY1),
+                             tc::smem_desc(ka + G::QK0_BYTES + k * 32, 8 * G::ROW1, G::LAY1), idesc_s, 1u);
+            tc::mma_commit(&s_full[t]);
+        };
+        auto issue_o = [&](int t, int vb) {                 // O_t = P_t V over the 128 keys in steps of 16
+            const uint32_t pa = p_base + t * G::P_BYTES, va = v_base + vb * G::V_BYTES, d = tmem_base + 256 + t * 128;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const uint32_t half = k >> 2, ko = (k & 3) * 32;
+                tc::mma_bf16(d, tc::smem_desc(pa + half * G::P_HALF + ko, 1024, 2),
+                             tc::smem_desc(va + half * G::V_HALF + ko, 1024, 2), idesc_o, k != 0);
+            }
+            tc::mma_commit(&o_full[t]);
+        };
+        bool ok = wait(bar_q, 0) && wait(bar_qz, 0) && wait(&k_full[0], 0);
+        if (ok) {
+            tc::tc_fence_after();
+            if (tc::elect_one()) {
+                for (int t = 0; t < nq; ++t) issue_s(t, 0);
+                tc::mma_commit(&k_empty[0]);
+            }
+            __syncwarp();
+        }
+        for (int j = 0; ok && j < nb; ++j) {
+            const int b = j & 1;
+            const uint32_t ph = (uint32_t)j & 1u, bph = (uint32_t)(j >> 1) & 1u;
+            for (int t = 0; ok && t < nq; ++t) {
+                ok = wait(&p_ready[t], ph);
+                if (ok && t == 0) ok = wait(&v_full[b], bph);
+                if (ok && j > 0) ok = wait(&o_free[t], ph ^ 1u);
+                if (!ok) break;
+                tc::tc_fence_after();
+                if (tc::elect_one()) {
+                    issue_o(t, b);
+                    if (t == nq - 1) tc::mma_commit(&v_empty[b]);
+                }
+                __syncwarp();
+                if (j + 1 < nb) {
+                    if (t == 0) { ok = wait(&k_full[b ^ 1], (uint32_t)((j + 1) >> 1) & 1u); if (!ok) break; tc::tc_fence_after(); }
+                    if (tc::elect_one()) {
+                        issue_s(t, b ^ 1);                  // S_t of the next block: this tile's softmax has consumed S_t
+                        if (t == nq - 1) tc::mma_commit(&k_empty[b ^ 1]);
+                    }
+                    __syncwarp();
+                }
+            }
+        }
+        if (!ok && lane == 0) fail();
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ softmax + output accumulation
+        const int t = warp >> 2, wq = warp & 3;
+        if (t < nq) {
+            const int r = wq * 32 + lane;                          // query row within the tile = TMEM lane
+            const uint32_t lane_sel = (uint32_t)(wq * 32) << 16;
+            const uint32_t tmem_S = tmem_base + t * 128 + lane_sel, tmem_O = tmem_base + 256 + t * 128 + lane_sel;
+            uint8_t* sQ = tiles + G::OFF_Q + t * G::QK_BYTES;
+            uint8_t* prow = tiles + G::OFF_P + t * G::P_BYTES + r * 128;
+            bool ok = wait(bar_q, 0);
+            if (ok) {
+                // zero the Q columns [d_head, d_pad) of this row (they belong to the next head)
+                if constexpr (G::W1 > 0) {
+                    constexpr int units = G::ROW1 / 16, rows_per_128 = 128 / G::ROW1;
+                    for (int u = (a.d_head - 64) / 8; u < units; ++u) {
+                        const int su = u ^ ((r / rows_per_128) & (units - 1));
+                        *reinterpret_cast<uint4*>(sQ + G::QK0_BYTES + r * G::ROW1 + su * 16) = make_uint4(0u, 0u, 0u, 0u);
+                    }
+                }
+                tc::fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(bar_qz);
+            }
+            float acc[DP];
+#pragma unroll
+            for (int c = 0; c < DP; ++c) acc[c] = 0.f;
+            float m_run = -INFINITY, l_run = 0.f, alpha_prev = 0.f;
+            const float cs = a.scale_log2e;
+            auto fold = [&](float alpha) {                          // acc = acc * alpha + O (the previous block's P V)
+#pragma unroll
+                for (int c0 = 0; c0 < DP; c0 += 16) {
+                    uint32_t v[16];
+                    tc::tmem_ld16(tmem_O + c0, v);
+                    tc::tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) acc[c0 + i] = fmaf(acc[c0 + i], alpha, __uint_as_float(v[i]));
+                }
+            };
+            for (int j = 0; ok && j < nb; ++j) {
+                const uint32_t ph = (uint32_t)j & 1u;
+                ok = wait(&s_full[t], ph);
+                if (!ok) break;
+                if (j > 0) {
+                    ok = wait(&o_full[t], ph ^ 1u);
+                    if (!ok) break;
+                    tc::tc_fence_after();
+                    fold(alpha_prev);
+                    tc::tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(&o_free[t]);
+                }
+                tc::tc_fence_after();
+                // pass 1: block maximum of this row
+                float mx = m_run;
+#pragma unroll
+                for (int c0 = 0; c0 < BKV; c0 += 32) {
+                    uint32_t v[32];
+                    tc::tmem_ld32(tmem_S + c0, v);
+                    tc::tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
+                }
+                const float alpha = ex2((m_run - mx) * cs);        // 0 on the first block (m_run = -inf)
+                const float mxc = mx * cs;
+                m_run = mx;
+                // pass 2: probabilities, row sum, bf16 P into shared memory (128-byte swizzled rows)
+                float sum = 0.f;
+#pragma unroll
+                for (int c0 = 0; c0 < BKV; c0 += 32) {
+                    uint32_t v[32];
+                    tc::tmem_ld32(tmem_S + c0, v);
+                    tc::tmem_wait_ld();
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float p0 = ex2(fmaf(__uint_as_float(v[2 * i]), cs, -mxc));
+                        const float p1 = ex2(fmaf(__uint_as_float(v[2 * i + 1]), cs, -mxc));
+                        sum += p0 + p1;
+                        __nv_bfloat162 bb = __floats2bfloat162_rn(p0, p1);
+                        pk[i] = *reinterpret_cast<uint32_t*>(&bb);
+                    }
+                    uint8_t* base = prow + (c0 >> 6) * G::P_HALF;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int unit = ((c0 & 63) >> 3) + u;      // 16-byte unit within the 128-byte row
+                        *reinterpret_cast<uint4*>(base + ((unit ^ (r & 7)) << 4)) = make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]);
+                    }
+                }
+                l_run = l_run * alpha + sum;
+                alpha_prev = alpha;
+                tc::tc_fence_before();
+                tc::fence_proxy_async();                            // P (generic-proxy stores) visible to the tensor core
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(&p_ready[t]);
+            }
+            if (ok) ok = wait(&o_full[t], (uint32_t)(nb - 1) & 1u);
+            if (ok) {
+                tc::tc_fence_after();
+                fold(alpha_prev);
+                const float inv = 1.f / l_run;
+                __nv_bfloat16* dst = a.out + ((long long)seq * T + q0 + t * BQ + r) * ((long long)a.heads * a.d_head) + (long long)head * a.d_head;
+                const int dh = a.d_head;                            // multiple of 8
+#pragma unroll
+                for (int c0 = 0; c0 < DP; c0 += 8) {
+                    if (c0 < dh) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            __nv_bfloat162 bb = __floats2bfloat162_rn(acc[c0 + 2 * i] * inv, acc[c0 + 2 * i + 1] * inv);
+                            w[i] = *reinterpret_cast<uint32_t*>(&bb);
+                        }
+                        *reinterpret_cast<uint4*>(dst + c0) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                }
+            } else if (lane == 0) {
+                fail();
+            }
+        }
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    if (warp == 9) { tc::tc_fence_after(); tc::tmem_dealloc(tmem_base, kTmemCols); }
+}
+
+template <int DP>
+int launch(int n_seq, int n_tok, int heads, int d_head, const void* qk, long long ld, int width, int q_col0, int k_col0,
+           const void* vt, void* out, uint32_t* err, cudaStream_t s) {
+    using G = Geo2<DP>;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [&] {
+        attr_err = cudaFuncSetAttribute(attention_tc2_kernel<DP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G::SMEM);
+    });
+    if (attr_err != cudaSuccess) return FREE_ERR_CUDA;
+    const uint64_t rows = (uint64_t)n_seq * n_tok, rows_v = (uint64_t)n_seq * heads * DP;
+    if (rows > 0x7fffffffull || rows_v > 0x7fffffffull) return FREE_ERR_SHAPE;
+    CUtensorMap mQK0, mQK1, mV;
+    FREE_TRY(free_tensor_map_2d(&mQK0, qk, (uint64_t)width, rows, (uint64_t)ld * 2, 64, 128, 128));
+    if (G::W1 > 0) FREE_TRY(free_tensor_map_2d(&mQK1, qk, (uint64_t)width, rows, (uint64_t)ld * 2, G::W1, 128, (int)G::ROW1));
+    else mQK1 = mQK0;
+    FREE_TRY(free_tensor_map_2d(&mV, vt, (uint64_t)n_tok, rows_v, (uint64_t)n_tok * 2, 64, DP, 128));
+    Attn2Args a{n_tok, heads, d_head, q_col0, k_col0, 1.4426950408889634f / sqrtf((float)d_head), (__nv_bfloat16*)out, err};
+    dim3 grid((n_tok + 2 * BQ - 1) / (2 * BQ), n_seq * heads);
+    attention_tc2_kernel<DP><<<grid, kThreads, G::SMEM, s>>>(mQK0, mQK1, mV, a);
+    return free_check_launch();
+}
+
+}  // namespace
+
+int attention_tc2_dpad(int d) { return d <= 64 ? 64 : (d <= 80 ? 80 : 96); }
+
+bool attention_tc2_supported(int n_tok, int d_head) {
+    return n_tok >= 128 && n_tok % 128 == 0 && d_head >= 64 && d_head % 8 == 0 && d_head <= 96;
+}
+
+int attention_tc2(int n_seq, int n_tok, int heads, int d_head, const void* qk, long long ld, int width, int q_col0, int k_col0,
+                  const void* vt, void* out, uint32_t* err, cudaStream_t s) {
+    if (n_seq < 1 || heads < 1 || !qk || !vt || !out || !err) return FREE_ERR_ARG;
+    if (!attention_tc2_supported(n_tok, d_head)) return FREE_ERR_UNSUPPORTED;
+    if (ld % 8 || q_col0 % 8 || k_col0 % 8 || width > ld || !free_aligned16(qk) || !free_aligned16(vt) || !free_aligned16(out)) return FREE_ERR_ALIGN;
+    const int dp = attention_tc2_dpad(d_head);
+    if ((long long)n_seq * heads > 65535) {
+        // grid.y limit: split the batch of sequences
+        const int per = 65535 / heads;
+        for (int s0 = 0; s0 < n_seq; s0 += per) {
+            const int ns = n_seq - s0 < per ? n_seq - s0 : per;
+            FREE_TRY(attention_tc2(ns, n_tok, heads, d_head, (const char*)qk + (size_t)s0 * n_tok * ld * 2, ld, width, q_col0, k_col0,
+                                   (const char*)vt + (size_t)s0 * heads * dp * n_tok * 2,
+                                   (char*)out + (size_t)s0 * n_tok * heads * d_head * 2, err, s));
+        }
+        return FREE_OK;
+    }
+    switch (dp) {
+        case 64: return launch<64>(n_seq, n_tok, heads, d_head, qk, ld, width, q_col0, k_col0, vt, out, err, s);
+        case 80: return launch<80>(n_seq, n_tok, heads, d_head, qk, ld, width, q_col0, k_col0, vt, out, err, s);
+        case 96: return launch<96>(n_seq, n_tok, heads, d_head, qk, ld, width, q_col0, k_col0, vt, out, err, s);
+        default: return FREE_ERR_UNSUPPORTED;
+    }
+}

@@ -23,6 +23,7 @@ struct free_ctx {
     free_drafter_desc dr;
     int n_tok, d_latent, patch_dim, out_dim, d_head, F;
     bool tc_attn;        // bf16 mode: attention on the tensor cores (else the CUDA-core kernel)
+    bool attn2;          // ... with the two-tile kernel that reads q and k token-major (needs D % 128 == 0, 64 <= d_head <= 96)
     int d_pad;
 };
 
@@ -81,7 +82,7 @@ Workspace plan(const free_ctx* c, int n, void* base) {
     w.x = (float*)take(M * D * 4);
     w.hn = take(M * D * 4);                       // fp32-sized: also holds the head's fp32 LayerNorm output
     const size_t qkv_tok = M * 3 * D * as;
-    const size_t qkv_head = c->tc_attn ? 3 * S * m.heads * (size_t)c->n_tok * c->d_pad * 2 : 0;
+    const size_t qkv_head = c->tc_attn ? 3 * S * m.heads * (size_t)c->n_tok * c->d_pad * 2 + 256 : 0;
     w.qkv = take(qkv_tok > qkv_head ? qkv_tok : qkv_head);
     w.att = take(M * D * as);
     w.hmlp = take(M * (size_t)c->F * as);
@@ -160,7 +161,15 @@ int run_blocks(const free_ctx* c, const Workspace& w, const Stack& st, int S, cu
         LinearArgs a; a.err = w.err;
         a.M = M; a.N = 3 * D; a.K = D; a.A = w.hn; a.W = wmat(st.bw.qkv_w, 3 * D); a.bias = st.bw.qkv_b + (size_t)i * 3 * D;
         a.out_dtype = m.dtype;
-        if (c->tc_attn) {
+        if (c->attn2) {
+            // q, k token-major [M, 2D]; v^T head-major behind them
+            a.epi = EPI_QKV_TOKV; a.heads = m.heads; a.d_head = c->d_head; a.d_pad = c->d_pad; a.n_tok = T;
+            a.out = w.qkv; a.ldo = 2LL * D; a.out_dtype = FREE_BF16;
+            a.vt = (char*)w.qkv + free_round_up((size_t)M * 2 * D * 2, 256);
+            { Scope p(c, PC_QKV, 2.0 * M * 3 * D * D, s); FREE_TRY(lin(c, a, s)); }
+            { Scope p(c, PC_ATTN, 4.0 * S * m.heads * (double)T * T * c->d_head, s);
+              FREE_TRY(attention_tc2(S, T, m.heads, c->d_head, w.qkv, 2LL * D, 2 * D, 0, D, a.vt, w.att, w.err, s)); }
+        } else if (c->tc_attn) {
             a.epi = EPI_QKV_HEADS; a.heads = m.heads; a.d_head = c->d_head; a.d_pad = c->d_pad; a.n_tok = T;
             const size_t per = (size_t)S * m.heads * T * c->d_pad * 2;
             a.q = w.qkv; a.k = (char*)w.qkv + per; a.vt = (char*)w.qkv + 2 * per;
@@ -408,6 +417,7 @@ extern "C" int free_create(const free_model_desc* t, const free_drafter_desc* d,
     c->d_head = t->D / t->heads;
     c->F = t->mlp_ratio * t->D;
     c->tc_attn = false;
+    c->attn2 = false;
     c->d_pad = c->d_head;
     if (t->dtype == FREE_BF16) {
         // tensor-core tiles need K % 64 == 0 and N % 16 == 0 for every GEMM of the stack
@@ -415,6 +425,7 @@ extern "C" int free_create(const free_model_desc* t, const free_drafter_desc* d,
             !linear_bf16_supported(c->F, t->D) || !linear_bf16_supported(t->D, c->F)) { delete c; return FREE_ERR_UNSUPPORTED; }
         c->tc_attn = attention_tc_supported(c->n_tok, c->d_head);
         if (c->tc_attn) c->d_pad = attention_tc_dpad(c->d_head);
+        c->attn2 = c->tc_attn && attention_tc2_supported(c->n_tok, c->d_head) && t->D % 128 == 0;
     }
     *out = c;
     return FREE_OK;

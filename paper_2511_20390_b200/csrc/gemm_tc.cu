@@ -312,6 +312,9 @@ static int validate_epilogue(const LinearArgs& l, long long ldo) {
         case EPI_QKV_HEADS:
             return (!l.q || !l.k || !l.vt || l.heads < 1 || l.d_head % 8 || l.d_pad % 8 || l.d_pad < l.d_head || l.n_tok < 1 ||
                     l.N != 3 * l.heads * l.d_head || l.M % l.n_tok) ? FREE_ERR_ARG : FREE_OK;
+        case EPI_QKV_TOKV:
+            return (!l.out || !l.vt || !free_aligned16(l.out) || ldo % 8 || l.heads < 1 || l.d_head % 8 || l.d_pad % 8 || l.d_pad < l.d_head ||
+                    l.n_tok < 1 || l.N != 3 * l.heads * l.d_head || l.M % l.n_tok) ? FREE_ERR_ARG : FREE_OK;
         default:
             return FREE_ERR_ARG;
     }
@@ -325,6 +328,7 @@ int linear_bf16(const LinearArgs& l, cudaStream_t s) {
     if (l.bias && !free_aligned16(l.bias)) return FREE_ERR_ALIGN;
     FREE_TRY(validate_epilogue(l, ldo));
     if (linear_bf16_pair_eligible(l)) return linear_bf16_pair(l, s);       // the large GEMMs: 256 x BN tiles on CTA pairs
+    if (l.epi == EPI_QKV_TOKV) return FREE_ERR_UNSUPPORTED;                // only the pair kernel has this epilogue
     TcArgs a{};
     a.M = l.M; a.N = l.N; a.K = l.K;
     a.BN = pick_bn(l.N);

@@ -20,8 +20,10 @@
 //              and clipped on the way out;
 //   warps 2-5  epilogue (both CTAs, each on its own 128 rows): tcgen05.ld, fused bias / GELU / gate, then
 //              through swizzled shared-memory staging to a TMA store, or a TMA add-reduction for the gated
-//              residual update (the fp32 residual stream is never read by the SM).  The QKV variant scatters
-//              straight into the head-major attention operands.
+//              residual update (the fp32 residual stream is never read by the SM).  QKV variants: HEADS scatters
+//              straight into head-major q, k, v^T; TOKV stores the q and k column blocks token-major like any
+//              other bf16 output and, for the v column blocks, stages groups of 8 columns transposed for all
+//              128 rows of the CTA and writes each group with one 2 KB TMA store into head-major v^T.
 // Tile order: N fastest, so the clusters in flight share a few row blocks of A while W stays in L2.
 #include "internal.h"
 #include "tc_common.cuh"
@@ -37,6 +39,8 @@ constexpr uint32_t kABytes = 128 * BK * 2;              // one CTA's A tile of a
 constexpr uint32_t kCtrlBytes = 1024;
 constexpr uint32_t kStageBufBytes = 4096;               // 32 rows x 128 bytes
 constexpr uint32_t kStagingBytes = 4 * 2 * kStageBufBytes;
+constexpr uint32_t kVBufBytes = 8192;                   // v^T staging: 3 buffers of 4 groups x (8 columns x 128 tokens)
+static_assert(3 * kVBufBytes <= kStagingBytes, "v^T staging must fit");
 constexpr uint32_t kSmemBudget = 227 * 1024;
 
 struct Tc2Args {
@@ -89,7 +93,7 @@ __device__ __forceinline__ void scatter_qkv(const Tc2Args& a, int row, int n0, c
 template <int EPI, bool OUT_BF16, int BN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapW,
-                  const __grid_constant__ CUtensorMap mapO, const Tc2Args a) {
+                  const __grid_constant__ CUtensorMap mapO, const __grid_constant__ CUtensorMap mapV, const Tc2Args a) {
     constexpr uint32_t kBBytes = (BN / 2) * BK * 2;          // one CTA's half of the W tile of a stage
     constexpr uint32_t kStageBytes = kABytes + kBBytes;
     extern __shared__ uint8_t smem_raw[];
@@ -98,7 +102,8 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
     uint64_t* empty = full + kMaxStages;
     uint64_t* accf = empty + kMaxStages;
     uint64_t* acce = accf + 2;                               // used in the even CTA only
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acce + 2);
+    uint64_t* ebar = acce + 2;                               // TOKV variant: meeting point of the four epilogue warps
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ebar + 1);
     volatile uint32_t* abort_flag = tmem_slot + 1;
     uint8_t* staging = smem + kCtrlBytes;
     uint8_t* tiles = staging + kStagingBytes;
@@ -112,6 +117,7 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
         for (int i = 0; i < 2; ++i) { tc::mbar_init(&accf[i], 1); tc::mbar_init(&acce[i], 8); }
+        tc::mbar_init(ebar, 4);
         *abort_flag = 0;
         tc::fence_barrier_init();
         tc::fence_proxy_async();
@@ -191,7 +197,15 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
         const uint32_t acce0 = tc::mapa(tc::smem_u32(&acce[0]), 0);
         uint8_t* my_stage = staging + (size_t)q * 2 * kStageBufBytes;
         constexpr int CH = OUT_BF16 ? 64 : 32;               // columns per staging buffer (128 bytes per row)
-        uint32_t tl = 0, nst = 0;
+        uint32_t tl = 0, nst = 0, eph = 0;
+        bool meet_ok = true;
+        auto meet = [&]() -> bool {                          // the four epilogue warps, bounded (unlike a named barrier)
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(ebar);
+            const bool met = tc::mbar_wait(ebar, eph);
+            eph ^= 1u;
+            return !__any_sync(0xffffffffu, !met);
+        };
         for (long long t = first; t < total; t += step, ++tl) {
             const int m_blk = (int)(t / a.num_n), n_blk = (int)(t % a.num_n);
             const uint32_t acc = tl & 1u, aph = (tl >> 1) & 1u;
@@ -219,6 +233,55 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
                         scatter_qkv(a, row, n0, v);
                     }
                 }
+            } else if (EPI == EPI_QKV_TOKV && n_blk * BN >= 2 * a.heads * a.d_head) {
+                // ---- a column block of v: transposed through shared memory into v^T [seq*heads*d_pad, n_tok]
+                // (mapV: box 128 tokens x 8 rows).  The CTA's 128 rows are 128 consecutive tokens of one sequence.
+                const int etid = q * 32 + lane;                         // row of the CTA tile = TMEM lane
+                const int row_base = m_blk * 256 + (int)rank * 128;
+                const bool live = row_base < a.M;
+                const int seq = live ? row_base / a.n_tok : 0, tok0 = live ? row_base % a.n_tok : 0;
+                // stores of the previous tile (which may have used the per-warp buffers) must have read their source
+                if (lane == 0) tc::bulk_wait_read<0>();
+                meet_ok = meet();
+                if (!meet_ok) { if (lane == 0) fail(FREE_DEV_ERR_ACC_FULL); break; }
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN && n_blk * BN + c0 < a.N; c0 += 32) {
+                    const int n0 = n_blk * BN + c0;
+                    uint32_t r[32];
+                    tc::tmem_ld32(t_addr + (uint32_t)c0, r);
+                    tc::tmem_wait_ld();
+                    uint8_t* buf = staging + (nst % 3u) * kVBufBytes;   // rewritten three chunks later, after two meetings
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float4 b = __ldg(reinterpret_cast<const float4*>(a.bias + n0) + i);
+                        const float v0 = __uint_as_float(r[4 * i + 0]) + b.x, v1 = __uint_as_float(r[4 * i + 1]) + b.y;
+                        const float v2 = __uint_as_float(r[4 * i + 2]) + b.z, v3 = __uint_as_float(r[4 * i + 3]) + b.w;
+                        uint8_t* gp = buf + (i >> 1) * 2048 + (i & 1) * 1024 + etid * 2;      // [group][column][token]
+                        *reinterpret_cast<__nv_bfloat16*>(gp) = __float2bfloat16(v0);
+                        *reinterpret_cast<__nv_bfloat16*>(gp + 256) = __float2bfloat16(v1);
+                        *reinterpret_cast<__nv_bfloat16*>(gp + 512) = __float2bfloat16(v2);
+                        *reinterpret_cast<__nv_bfloat16*>(gp + 768) = __float2bfloat16(v3);
+                    }
+                    tc::fence_proxy_async();
+                    meet_ok = meet();
+                    if (!meet_ok) { if (lane == 0) fail(FREE_DEV_ERR_ACC_FULL); break; }
+                    if (lane == 0) {                                    // each warp issues one of the four groups
+                        if (live) {
+                            const int g = warp - 2;
+                            const int vc = n0 + 8 * g - 2 * a.heads * a.d_head;
+                            const int hd = vc / a.d_head, c = vc % a.d_head;
+                            tc::tma_store_2d(&mapV, tc::smem_u32(buf + g * 2048), tok0, (seq * a.heads + hd) * a.d_pad + c);
+                        }
+                        tc::bulk_commit();
+                        tc::bulk_wait_read<1>();
+                    }
+                    ++nst;
+                }
+                if (!meet_ok) break;
+                // the next tile may use the per-warp buffers: this tile's stores must have read theirs first
+                if (lane == 0) tc::bulk_wait_read<0>();
+                meet_ok = meet();
+                if (!meet_ok) { if (lane == 0) fail(FREE_DEV_ERR_ACC_FULL); break; }
             } else {
                 const int rowc = row < a.M ? row : a.M - 1;
                 const float* gp = (EPI == EPI_GATE_RESIDUAL && a.gate) ? a.gate + (long long)(rowc / a.rows_per_seq) * a.gate_stride : nullptr;
@@ -302,7 +365,8 @@ int sm_count() {
 }
 
 template <int EPI, bool OUT_BF16, int BN>
-int launch(const CUtensorMap& mA, const CUtensorMap& mW, const CUtensorMap& mO, const Tc2Args& a, size_t smem, cudaStream_t s) {
+int launch(const CUtensorMap& mA, const CUtensorMap& mW, const CUtensorMap& mO, const CUtensorMap& mV, const Tc2Args& a, size_t smem,
+           cudaStream_t s) {
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] {
@@ -312,7 +376,7 @@ int launch(const CUtensorMap& mA, const CUtensorMap& mW, const CUtensorMap& mO, 
     const long long tiles = (long long)a.num_m * a.num_n;
     const long long pairs = sm_count() / 2;
     const int grid = 2 * (int)(tiles < pairs ? tiles : pairs);
-    linear_tc2_kernel<EPI, OUT_BF16, BN><<<grid, kThreads, smem, s>>>(mA, mW, mO, a);
+    linear_tc2_kernel<EPI, OUT_BF16, BN><<<grid, kThreads, smem, s>>>(mA, mW, mO, mV, a);
     return free_check_launch();
 }
 
@@ -331,16 +395,24 @@ int dispatch(const LinearArgs& l, Tc2Args a, cudaStream_t s) {
     switch (l.epi) {
         case EPI_BIAS:
             FREE_TRY(free_tensor_map_2d_typed(&mO, ob ? 2 : 4, l.out, (uint64_t)l.N, (uint64_t)l.M, (uint64_t)ldo * (ob ? 2 : 4), ob ? 64 : 32, 32, 128));
-            return ob ? launch<EPI_BIAS, true, BN>(mA, mW, mO, a, smem, s) : launch<EPI_BIAS, false, BN>(mA, mW, mO, a, smem, s);
+            return ob ? launch<EPI_BIAS, true, BN>(mA, mW, mO, mO, a, smem, s) : launch<EPI_BIAS, false, BN>(mA, mW, mO, mO, a, smem, s);
         case EPI_BIAS_GELU:
             FREE_TRY(free_tensor_map_2d_typed(&mO, 2, l.out, (uint64_t)l.N, (uint64_t)l.M, (uint64_t)ldo * 2, 64, 32, 128));
-            return launch<EPI_BIAS_GELU, true, BN>(mA, mW, mO, a, smem, s);
+            return launch<EPI_BIAS_GELU, true, BN>(mA, mW, mO, mO, a, smem, s);
         case EPI_GATE_RESIDUAL:
             FREE_TRY(free_tensor_map_2d_typed(&mO, 4, l.resid, (uint64_t)l.N, (uint64_t)l.M, (uint64_t)l.N * 4, 32, 32, 128));
-            return launch<EPI_GATE_RESIDUAL, false, BN>(mA, mW, mO, a, smem, s);
+            return launch<EPI_GATE_RESIDUAL, false, BN>(mA, mW, mO, mO, a, smem, s);
         case EPI_QKV_HEADS:
             mO = mA;                                         // unused by this variant
-            return launch<EPI_QKV_HEADS, true, BN>(mA, mW, mO, a, smem, s);
+            return launch<EPI_QKV_HEADS, true, BN>(mA, mW, mO, mO, a, smem, s);
+        case EPI_QKV_TOKV: {
+            CUtensorMap mV;
+            const int qk_cols = 2 * l.heads * l.d_head;
+            FREE_TRY(free_tensor_map_2d_typed(&mO, 2, l.out, (uint64_t)qk_cols, (uint64_t)l.M, (uint64_t)ldo * 2, 64, 32, 128));
+            FREE_TRY(free_tensor_map_2d_typed(&mV, 2, l.vt, (uint64_t)l.n_tok, (uint64_t)(l.M / l.n_tok) * l.heads * l.d_pad,
+                                              (uint64_t)l.n_tok * 2, 128, 8, 0));
+            return launch<EPI_QKV_TOKV, true, BN>(mA, mW, mO, mV, a, smem, s);
+        }
         default:
             return FREE_ERR_UNSUPPORTED;
     }
@@ -350,13 +422,15 @@ int dispatch(const LinearArgs& l, Tc2Args a, cudaStream_t s) {
 
 // Shapes and epilogues the pair kernel takes; everything else stays on the single-CTA kernel.
 bool linear_bf16_pair_eligible(const LinearArgs& l) {
-    if (l.M <= 128 || l.K < BK || l.K % BK) return false;
+    if ((l.M <= 128 && l.epi != EPI_QKV_TOKV) || l.K < BK || l.K % BK) return false;
     if (l.N < 256 || l.N % 64) return false;            // column chunks of the epilogue are 64 wide
     switch (l.epi) {
         case EPI_BIAS: return l.out != nullptr;
         case EPI_BIAS_GELU: return l.out != nullptr && l.out_dtype == FREE_BF16;
         case EPI_GATE_RESIDUAL: return l.resid != nullptr;
         case EPI_QKV_HEADS: return l.bias != nullptr;
+        case EPI_QKV_TOKV:                                   // column blocks are wholly q/k or wholly v; 128-row blocks lie in one sequence
+            return l.bias != nullptr && (2 * l.heads * l.d_head) % 256 == 0 && l.n_tok % 128 == 0;
         default: return false;
     }
 }

@@ -11,6 +11,7 @@ enum {
     EPI_GATE_RESIDUAL = FREE_EPI_GATE_RESIDUAL,   // resid += gate * (acc + bias); gate == nullptr means 1
     EPI_BIAS_EMB_SILU = 4,                        // out = silu(acc + bias + emb[emb_idx[row], n])
     EPI_QKV_HEADS = 5,                            // bf16 only: scatter (acc + bias) into head-major q, k and v^T
+    EPI_QKV_TOKV = 6,                             // bf16 only (CTA-pair kernel): q and k token-major into out[M, 2D], v^T head-major
 };
 
 struct LinearArgs {
@@ -44,6 +45,12 @@ int attention_tc(int n_seq, int n_tok, int heads, int d_head, int d_pad, const v
                  void* out, uint32_t* err, cudaStream_t s);
 bool attention_tc_supported(int n_tok, int d_head);
 int attention_tc_dpad(int d_head);
+// Two query tiles per CTA; q and k read from a token-major matrix [n_seq*n_tok, ld] (first `width` columns valid),
+// head h of q at column q_col0 + h*d_head, of k at k_col0 + h*d_head; vt [n_seq, heads, d_pad, n_tok].
+int attention_tc2(int n_seq, int n_tok, int heads, int d_head, const void* qk, long long ld, int width, int q_col0, int k_col0,
+                  const void* vt, void* out, uint32_t* err, cudaStream_t s);
+bool attention_tc2_supported(int n_tok, int d_head);
+int attention_tc2_dpad(int d_head);
 
 // ---- elementwise / row kernels ----------------------------------------------------------------
 int cond_setup(int dtype, int n_states, int G, int freq_dim, int n_classes, int N_sched,

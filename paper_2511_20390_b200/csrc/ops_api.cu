@@ -24,6 +24,18 @@ __global__ void repack_qkv_kernel(int n_seq, int n_tok, int heads, int dh, int d
     }
 }
 
+// v of token-major qkv [n_seq, n_tok, 3, heads, d_head] -> v^T [n_seq, heads, d_pad, n_tok] (zero padded)
+__global__ void repack_vt_kernel(int n_seq, int n_tok, int heads, int dh, int dp, const __nv_bfloat16* qkv, __nv_bfloat16* vt) {
+    const long long total = (long long)n_seq * heads * dp * n_tok;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const int t = (int)(i % n_tok);
+        const int c = (int)((i / n_tok) % dp);
+        const int h = (int)((i / ((long long)n_tok * dp)) % heads);
+        const int s = (int)(i / ((long long)n_tok * dp * heads));
+        vt[i] = c < dh ? qkv[(((long long)s * n_tok + t) * 3 + 2) * heads * dh + (long long)h * dh + c] : __float2bfloat16(0.f);
+    }
+}
+
 }  // namespace
 
 extern "C" size_t free_op_linear_workspace_bytes(void) { return 256; }
@@ -64,6 +76,17 @@ extern "C" int free_op_attention(int dtype, int n_seq, int n_tok, int heads, int
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     if (dtype == FREE_FP32 || !attention_tc_supported(n_tok, d_head))
         return attention_simt(dtype, n_seq, n_tok, heads, d_head, qkv, out, s);
+    if (attention_tc2_supported(n_tok, d_head)) {
+        // the two-tile kernel reads q and k from the caller's matrix as it is; only v^T is prepared
+        const int dp2 = attention_tc2_dpad(d_head);
+        __nv_bfloat16* vt2 = (__nv_bfloat16*)((char*)ws + 256);
+        const long long tot = (long long)n_seq * heads * n_tok * dp2;
+        const unsigned g2 = (unsigned)((tot + 255) / 256 > 148 * 16 ? 148 * 16 : (tot + 255) / 256);
+        repack_vt_kernel<<<g2, 256, 0, s>>>(n_seq, n_tok, heads, d_head, dp2, (const __nv_bfloat16*)qkv, vt2);
+        FREE_TRY(free_check_launch());
+        const int D = heads * d_head;
+        return attention_tc2(n_seq, n_tok, heads, d_head, qkv, 3LL * D, 3 * D, 0, D, vt2, out, reinterpret_cast<uint32_t*>(ws), s);
+    }
     const int dp = attention_tc_dpad(d_head);
     const size_t per = free_round_up((size_t)n_seq * heads * n_tok * dp * 2, 256);
     char* base = (char*)ws + 256;

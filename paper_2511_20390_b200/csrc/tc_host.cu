@@ -38,7 +38,9 @@ int free_tensor_map_2d_typed(CUtensorMap* map, int elem_bytes, const void* base,
     auto fn = encode_fn();
     if (!fn) return FREE_ERR_CUDA;
     if (elem_bytes != 2 && elem_bytes != 4) return FREE_ERR_ARG;
-    if (box_inner * (uint32_t)elem_bytes > (uint32_t)swizzle_bytes || box_outer > 256 || outer_stride_bytes % 16) return FREE_ERR_UNSUPPORTED;
+    // swizzle_bytes 0: no swizzle (the box's inner extent is then only limited to 256 elements)
+    if ((swizzle_bytes ? box_inner * (uint32_t)elem_bytes > (uint32_t)swizzle_bytes : box_inner > 256) ||
+        (box_inner * (uint32_t)elem_bytes) % 16 || box_outer > 256 || outer_stride_bytes % 16) return FREE_ERR_UNSUPPORTED;
     cuuint64_t dims[2] = {inner, outer};
     cuuint64_t strides[1] = {outer_stride_bytes};
     cuuint32_t box[2] = {box_inner, box_outer};
