@@ -7,10 +7,13 @@
 //   warp 8      TMA producer: Q tiles once, then K and V^T blocks of 128 keys into double buffers
 //   warp 9      MMA issuer (the warp runs converged, one elected lane issues):
 //               S_t = Q_t K^T (128 x 128 x d_pad) into TMEM, O_t = P_t V (128 x d_pad x 128) into TMEM
-// Per block of 128 keys and per tile: wait S, fold the previous block's O into the fp32 register accumulator
-// (rescaled by the running-max correction), two passes over S in TMEM (row maximum; exp2, row sum, P rounded to
-// bf16 and stored to shared memory in the MMA operand layout), signal P.  The issue order
-// PV_0, S_0(next), PV_1, S_1(next) keeps one tile's MMAs in flight while the other tile is in its softmax.
+// Per block of 128 keys and per tile, a softmax thread pulls its whole row of S out of TMEM in one round trip and
+// releases S at once (the next block's S is issued while this softmax still runs), takes the row maximum, turns the
+// row into exp2 probabilities (row sum in fp32, P rounded to bf16 into shared memory in the MMA operand layout) and
+// signals P.  O_t accumulates in TMEM across all key blocks: the exponent offset of a row is only moved when the row
+// maximum has grown by more than 8 (a factor 256), in which case the row's O and running sum are rescaled in place
+// before that block's P V is issued; numerator and denominator always share the offset, so the result is exact.
+// Issue order per block: S_0(next), PV_0, S_1(next), PV_1.
 //
 // Operands.  q and k are read straight from a token-major bf16 matrix [n_seq * n_tok, ld] (the output of the QKV
 // linear layer): head h of q starts at column q_col0 + h * d_head, of k at k_col0 + h * d_head.  d_pad is 64 plus a
@@ -75,7 +78,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
     uint64_t* s_full = bar_q + 10;      // [2] per tile: S complete
     uint64_t* p_ready = bar_q + 12;     // [2] per tile: P stored and S consumed (4 warp arrivals)
     uint64_t* o_full = bar_q + 14;      // [2] per tile: O_j complete
-    uint64_t* o_free = bar_q + 16;      // [2] per tile: O_j folded into registers (4 warp arrivals)
+    uint64_t* s_free = bar_q + 16;      // [2] per tile: S_j read out of TMEM (4 warp arrivals)
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_q + 18);
     volatile uint32_t* abort_flag = tmem_slot + 1;
     uint8_t* tiles = smem + 1024;
@@ -91,7 +94,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
         tc::mbar_init(bar_q, 1); tc::mbar_init(bar_qz, 4 * nq);
         for (int i = 0; i < 2; ++i) {
             tc::mbar_init(&k_full[i], 1); tc::mbar_init(&k_empty[i], 1); tc::mbar_init(&v_full[i], 1); tc::mbar_init(&v_empty[i], 1);
-            tc::mbar_init(&s_full[i], 1); tc::mbar_init(&p_ready[i], 4); tc::mbar_init(&o_full[i], 1); tc::mbar_init(&o_free[i], 4);
+            tc::mbar_init(&s_full[i], 1); tc::mbar_init(&p_ready[i], 4); tc::mbar_init(&o_full[i], 1); tc::mbar_init(&s_free[i], 4);
         }
         *abort_flag = 0;
         tc::fence_barrier_init();
@@ -168,13 +171,13 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
                              tc::smem_desc(ka + G::QK0_BYTES + k * 32, 8 * G::ROW1, G::LAY1), idesc_s, 1u);
             tc::mma_commit(&s_full[t]);
         };
-        auto issue_o = [&](int t, int vb) {                 // O_t = P_t V over the 128 keys in steps of 16
+        auto issue_o = [&](int t, int vb, uint32_t accumulate) {   // O_t (+)= P_t V over the 128 keys in steps of 16
             const uint32_t pa = p_base + t * G::P_BYTES, va = v_base + vb * G::V_BYTES, d = tmem_base + 256 + t * 128;
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
                 const uint32_t half = k >> 2, ko = (k & 3) * 32;
                 tc::mma_bf16(d, tc::smem_desc(pa + half * G::P_HALF + ko, 1024, 2),
-                             tc::smem_desc(va + half * G::V_HALF + ko, 1024, 2), idesc_o, k != 0);
+                             tc::smem_desc(va + half * G::V_HALF + ko, 1024, 2), idesc_o, (accumulate | (uint32_t)k) != 0 ? 1u : 0u);
             }
             tc::mma_commit(&o_full[t]);
         };
@@ -191,24 +194,27 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
             const int b = j & 1;
             const uint32_t ph = (uint32_t)j & 1u, bph = (uint32_t)(j >> 1) & 1u;
             for (int t = 0; ok && t < nq; ++t) {
-                ok = wait(&p_ready[t], ph);
-                if (ok && t == 0) ok = wait(&v_full[b], bph);
-                if (ok && j > 0) ok = wait(&o_free[t], ph ^ 1u);
-                if (!ok) break;
-                tc::tc_fence_after();
-                if (tc::elect_one()) {
-                    issue_o(t, b);
-                    if (t == nq - 1) tc::mma_commit(&v_empty[b]);
-                }
-                __syncwarp();
                 if (j + 1 < nb) {
-                    if (t == 0) { ok = wait(&k_full[b ^ 1], (uint32_t)((j + 1) >> 1) & 1u); if (!ok) break; tc::tc_fence_after(); }
+                    // S_t of the next block as soon as this tile's softmax has pulled S_t of this block out of TMEM
+                    ok = wait(&s_free[t], ph);
+                    if (ok && t == 0) ok = wait(&k_full[b ^ 1], (uint32_t)((j + 1) >> 1) & 1u);
+                    if (!ok) break;
+                    tc::tc_fence_after();
                     if (tc::elect_one()) {
-                        issue_s(t, b ^ 1);                  // S_t of the next block: this tile's softmax has consumed S_t
+                        issue_s(t, b ^ 1);
                         if (t == nq - 1) tc::mma_commit(&k_empty[b ^ 1]);
                     }
                     __syncwarp();
                 }
+                ok = wait(&p_ready[t], ph);
+                if (ok && t == 0) ok = wait(&v_full[b], bph);
+                if (!ok) break;
+                tc::tc_fence_after();
+                if (tc::elect_one()) {
+                    issue_o(t, b, j > 0 ? 1u : 0u);
+                    if (t == nq - 1) tc::mma_commit(&v_empty[b]);
+                }
+                __syncwarp();
             }
         }
         if (!ok && lane == 0) fail();
@@ -236,61 +242,64 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(bar_qz);
             }
-            float acc[DP];
-#pragma unroll
-            for (int c = 0; c < DP; ++c) acc[c] = 0.f;
-            float m_run = -INFINITY, l_run = 0.f, alpha_prev = 0.f;
+            float m_used = -INFINITY, l_run = 0.f;                  // exponent offset of this row and its running sum
             const float cs = a.scale_log2e;
-            auto fold = [&](float alpha) {                          // acc = acc * alpha + O (the previous block's P V)
-#pragma unroll
-                for (int c0 = 0; c0 < DP; c0 += 16) {
-                    uint32_t v[16];
-                    tc::tmem_ld16(tmem_O + c0, v);
-                    tc::tmem_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) acc[c0 + i] = fmaf(acc[c0 + i], alpha, __uint_as_float(v[i]));
-                }
-            };
             for (int j = 0; ok && j < nb; ++j) {
                 const uint32_t ph = (uint32_t)j & 1u;
                 ok = wait(&s_full[t], ph);
                 if (!ok) break;
-                if (j > 0) {
+                tc::tc_fence_after();
+                uint32_t sv[128];                                   // the whole row of S: one TMEM round trip
+                tc::tmem_ld64(tmem_S, *reinterpret_cast<uint32_t(*)[64]>(&sv[0]));
+                tc::tmem_ld64(tmem_S + 64, *reinterpret_cast<uint32_t(*)[64]>(&sv[64]));
+                tc::tmem_wait_ld();
+                tc::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(&s_free[t]);         // the next block's S may overwrite TMEM now
+                float m0 = __uint_as_float(sv[0]), m1 = __uint_as_float(sv[1]), m2 = __uint_as_float(sv[2]), m3 = __uint_as_float(sv[3]);
+#pragma unroll
+                for (int i = 4; i < 128; i += 4) {
+                    m0 = fmaxf(m0, __uint_as_float(sv[i])); m1 = fmaxf(m1, __uint_as_float(sv[i + 1]));
+                    m2 = fmaxf(m2, __uint_as_float(sv[i + 2])); m3 = fmaxf(m3, __uint_as_float(sv[i + 3]));
+                }
+                const float m_new = fmaxf(m_used, fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)));
+                bool waited_o = false;
+                if (__any_sync(0xffffffffu, (m_new - m_used) * cs > 8.f)) {
+                    // move the exponent offset of the rows of this warp (always on the first block)
+                    if (j > 0) {
+                        ok = wait(&o_full[t], ph ^ 1u);             // O_t complete up to the previous block
+                        if (!ok) break;
+                        waited_o = true;
+                        tc::tc_fence_after();
+                        const float alpha = ex2((m_used - m_new) * cs);
+#pragma unroll
+                        for (int c0 = 0; c0 < DP; c0 += 16) {
+                            uint32_t ov[16];
+                            tc::tmem_ld16(tmem_O + c0, ov);
+                            tc::tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+                            tc::tmem_st16(tmem_O + c0, ov);
+                        }
+                        tc::tmem_wait_st();
+                        l_run *= alpha;
+                    }
+                    m_used = m_new;
+                }
+                if (j > 0 && !waited_o) {                           // the previous P V has read P: the buffer is free
                     ok = wait(&o_full[t], ph ^ 1u);
                     if (!ok) break;
-                    tc::tc_fence_after();
-                    fold(alpha_prev);
-                    tc::tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) tc::mbar_arrive(&o_free[t]);
                 }
-                tc::tc_fence_after();
-                // pass 1: block maximum of this row
-                float mx = m_run;
+                const float mc = m_used * cs;
+                float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
                 for (int c0 = 0; c0 < BKV; c0 += 32) {
-                    uint32_t v[32];
-                    tc::tmem_ld32(tmem_S + c0, v);
-                    tc::tmem_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
-                }
-                const float alpha = ex2((m_run - mx) * cs);        // 0 on the first block (m_run = -inf)
-                const float mxc = mx * cs;
-                m_run = mx;
-                // pass 2: probabilities, row sum, bf16 P into shared memory (128-byte swizzled rows)
-                float sum = 0.f;
-#pragma unroll
-                for (int c0 = 0; c0 < BKV; c0 += 32) {
-                    uint32_t v[32];
-                    tc::tmem_ld32(tmem_S + c0, v);
-                    tc::tmem_wait_ld();
                     uint32_t pk[16];
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
-                        const float p0 = ex2(fmaf(__uint_as_float(v[2 * i]), cs, -mxc));
-                        const float p1 = ex2(fmaf(__uint_as_float(v[2 * i + 1]), cs, -mxc));
-                        sum += p0 + p1;
+                        const float p0 = ex2(fmaf(__uint_as_float(sv[c0 + 2 * i]), cs, -mc));
+                        const float p1 = ex2(fmaf(__uint_as_float(sv[c0 + 2 * i + 1]), cs, -mc));
+                        sum0 += p0; sum1 += p1;
                         __nv_bfloat162 bb = __floats2bfloat162_rn(p0, p1);
                         pk[i] = *reinterpret_cast<uint32_t*>(&bb);
                     }
@@ -301,8 +310,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
                         *reinterpret_cast<uint4*>(base + ((unit ^ (r & 7)) << 4)) = make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]);
                     }
                 }
-                l_run = l_run * alpha + sum;
-                alpha_prev = alpha;
+                l_run += sum0 + sum1;
                 tc::tc_fence_before();
                 tc::fence_proxy_async();                            // P (generic-proxy stores) visible to the tensor core
                 __syncwarp();
@@ -311,20 +319,25 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
             if (ok) ok = wait(&o_full[t], (uint32_t)(nb - 1) & 1u);
             if (ok) {
                 tc::tc_fence_after();
-                fold(alpha_prev);
                 const float inv = 1.f / l_run;
                 __nv_bfloat16* dst = a.out + ((long long)seq * T + q0 + t * BQ + r) * ((long long)a.heads * a.d_head) + (long long)head * a.d_head;
                 const int dh = a.d_head;                            // multiple of 8
 #pragma unroll
-                for (int c0 = 0; c0 < DP; c0 += 8) {
-                    if (c0 < dh) {
-                        uint32_t w[4];
+                for (int c0 = 0; c0 < DP; c0 += 16) {
+                    uint32_t ov[16];
+                    tc::tmem_ld16(tmem_O + c0, ov);
+                    tc::tmem_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            __nv_bfloat162 bb = __floats2bfloat162_rn(acc[c0 + 2 * i] * inv, acc[c0 + 2 * i + 1] * inv);
-                            w[i] = *reinterpret_cast<uint32_t*>(&bb);
+                    for (int h8 = 0; h8 < 16; h8 += 8) {
+                        if (c0 + h8 < dh) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                __nv_bfloat162 bb = __floats2bfloat162_rn(__uint_as_float(ov[h8 + 2 * i]) * inv, __uint_as_float(ov[h8 + 2 * i + 1]) * inv);
+                                w[i] = *reinterpret_cast<uint32_t*>(&bb);
+                            }
+                            *reinterpret_cast<uint4*>(dst + c0 + h8) = make_uint4(w[0], w[1], w[2], w[3]);
                         }
-                        *reinterpret_cast<uint4*>(dst + c0) = make_uint4(w[0], w[1], w[2], w[3]);
                     }
                 }
             } else if (lane == 0) {
