@@ -2,15 +2,19 @@
 //
 // One CTA (one per SM) owns 256 queries of one (sequence, head): two tiles of 128 queries that alternate on the
 // tensor core, so that the softmax of one tile runs while the MMAs of the other execute.
-//   warps 0-3   softmax + output accumulation of query tile 0 (thread = one query row = one TMEM lane)
-//   warps 4-7   the same for query tile 1
-//   warp 8      TMA producer: Q tiles once, then K and V^T blocks of 128 keys into double buffers
-//   warp 9      MMA issuer (the warp runs converged, one elected lane issues):
+//   warps 0-7   softmax of query tile 0: a query row (= one TMEM lane) is shared by two threads, warp w and warp
+//               w + 4, which take the two halves of 64 keys of every block (four softmax warps per scheduler keep
+//               the exp2 unit, which bounds this kernel at d_head 72, fed while others wait on TMEM or barriers)
+//   warps 8-15  the same for query tile 1
+//   warp 16     TMA producer: Q tiles once, then K and V^T blocks of 128 keys into double buffers
+//   warps 17-18 MMA issuers, one per query tile (each runs converged, one elected lane issues; a barrier poll costs
+//               ~200 clocks and an MMA issue ~50-100, so one warp serving both tiles was the bottleneck):
 //               S_t = Q_t K^T (128 x 128 x d_pad) into TMEM, O_t = P_t V (128 x d_pad x 128) into TMEM
-// Per block of 128 keys and per tile, a softmax thread pulls its whole row of S out of TMEM in one round trip and
+// Per block of 128 keys and per tile, a softmax thread pulls its half row of S out of TMEM in one round trip and
 // releases S at once (the next block's S is issued while this softmax still runs), takes the row maximum, turns the
 // row into exp2 probabilities (row sum in fp32, P rounded to bf16 into shared memory in the MMA operand layout) and
-// signals P.  O_t accumulates in TMEM across all key blocks: the exponent offset of a row is only moved when the row
+// signals P; the two threads of a row exchange their half-row maxima through shared memory so that both use the same
+// exponent offset, and add their partial row sums at the end.  O_t accumulates in TMEM across all key blocks: the exponent offset of a row is only moved when the row
 // maximum has grown by more than 8 (a factor 256), in which case the row's O and running sum are rescaled in place
 // before that block's P V is issued; numerator and denominator always share the offset, so the result is exact.
 // Issue order per block: S_0(next), PV_0, S_1(next), PV_1.
@@ -28,7 +32,8 @@
 namespace {
 
 constexpr int BQ = 128, BKV = 128;
-constexpr int kThreads = 320;
+constexpr int kThreads = 608;
+constexpr uint32_t kCtrlBytes = 8192;          // barriers (1 KB), row-maximum exchange (4 KB), row-sum exchange (2 KB)
 constexpr uint32_t kTmemCols = 512;           // S_0 [0,128), S_1 [128,256), O_0 [256,384), O_1 [384,512)
 
 struct Attn2Args {
@@ -55,7 +60,7 @@ template <int DP> struct Geo2 {
     static constexpr uint32_t OFF_V = OFF_K + 2 * QK_BYTES;             // two buffers
     static constexpr uint32_t OFF_P = OFF_V + 2 * V_BYTES;              // two tiles
     static constexpr uint32_t TILE_BYTES = OFF_P + 2 * P_BYTES;
-    static constexpr uint32_t SMEM = 1024 /*align*/ + 1024 /*barriers*/ + TILE_BYTES;
+    static constexpr uint32_t SMEM = 1024 /*align*/ + kCtrlBytes + TILE_BYTES;
     static_assert(QK_BYTES % 1024 == 0 && V_HALF % 1024 == 0, "tiles must keep the swizzle alignment");
     static_assert(SMEM <= 227 * 1024, "does not fit in shared memory");
 };
@@ -79,9 +84,12 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
     uint64_t* p_ready = bar_q + 12;     // [2] per tile: P stored and S consumed (4 warp arrivals)
     uint64_t* o_full = bar_q + 14;      // [2] per tile: O_j complete
     uint64_t* s_free = bar_q + 16;      // [2] per tile: S_j read out of TMEM (4 warp arrivals)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_q + 18);
+    uint64_t* pair_bar = bar_q + 18;    // [8] tile * 4 + lane quarter: the two warps that share rows (2 arrivals)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_q + 26);
     volatile uint32_t* abort_flag = tmem_slot + 1;
-    uint8_t* tiles = smem + 1024;
+    float* mx_x = reinterpret_cast<float*>(smem + 1024);       // [parity][tile][half][row]
+    float* l_x = reinterpret_cast<float*>(smem + 5120);        // [tile][half][row]
+    uint8_t* tiles = smem + kCtrlBytes;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int sh = blockIdx.y;                              // sequence * heads + head
@@ -92,15 +100,16 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
 
     if (threadIdx.x == 0) {
         tc::mbar_init(bar_q, 1); tc::mbar_init(bar_qz, 4 * nq);
+        for (int i = 0; i < 8; ++i) tc::mbar_init(&pair_bar[i], 2);
         for (int i = 0; i < 2; ++i) {
-            tc::mbar_init(&k_full[i], 1); tc::mbar_init(&k_empty[i], 1); tc::mbar_init(&v_full[i], 1); tc::mbar_init(&v_empty[i], 1);
-            tc::mbar_init(&s_full[i], 1); tc::mbar_init(&p_ready[i], 4); tc::mbar_init(&o_full[i], 1); tc::mbar_init(&s_free[i], 4);
+            tc::mbar_init(&k_full[i], 1); tc::mbar_init(&k_empty[i], nq); tc::mbar_init(&v_full[i], 1); tc::mbar_init(&v_empty[i], nq);
+            tc::mbar_init(&s_full[i], 1); tc::mbar_init(&p_ready[i], 8); tc::mbar_init(&o_full[i], 1); tc::mbar_init(&s_free[i], 8);
         }
         *abort_flag = 0;
         tc::fence_barrier_init();
         tc::fence_proxy_async();
     }
-    if (warp == 9) { tc::tmem_alloc(tmem_slot, kTmemCols); tc::tmem_relinquish(); }
+    if (warp == 17) { tc::tmem_alloc(tmem_slot, kTmemCols); tc::tmem_relinquish(); }
     tc::tc_fence_before();
     __syncthreads();
     tc::tc_fence_after();
@@ -110,8 +119,16 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
     auto wait = [&](uint64_t* bar, uint32_t parity) -> bool {
         return __all_sync(0xffffffffu, !*abort_flag && tc::mbar_wait(bar, parity));
     };
+    // two barriers polled together (their poll latencies overlap)
+    auto wait2 = [&](uint64_t* b0, uint32_t p0, uint64_t* b1, uint32_t p1) -> bool {
+        if (*abort_flag) return false;
+        bool r0 = tc::mbar_try_wait(b0, p0), r1 = tc::mbar_try_wait(b1, p1);
+        if (!r0) r0 = tc::mbar_wait(b0, p0);
+        if (!r1) r1 = tc::mbar_wait(b1, p1);
+        return __all_sync(0xffffffffu, r0 && r1);
+    };
 
-    if (warp == 8) {
+    if (warp == 16) {
         // ------------------------------------------------------------------ TMA producer
         const int row_q = seq * T + q0;                     // row of the first query in the token-major matrix
         const int xq = a.q_col0 + head * a.d_head, xk = a.k_col0 + head * a.d_head;
@@ -155,131 +172,150 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
             while (clock64() - t0 < 400000ll) { }
         }
         __syncwarp();
-    } else if (warp == 9) {
-        // ------------------------------------------------------------------ MMA issuer
-        const uint32_t idesc_s = tc::idesc_bf16(BQ, BKV), idesc_o = tc::idesc_bf16(BQ, DP);
-        const uint32_t q_base = tc::smem_u32(tiles + G::OFF_Q), k_base = tc::smem_u32(tiles + G::OFF_K);
-        const uint32_t v_base = tc::smem_u32(tiles + G::OFF_V), p_base = tc::smem_u32(tiles + G::OFF_P);
-        auto issue_s = [&](int t, int kb) {                 // S_t = Q_t K^T over d_pad in steps of 16 (elected lane)
-            const uint32_t qa = q_base + t * G::QK_BYTES, ka = k_base + kb * G::QK_BYTES, d = tmem_base + t * 128;
+    } else if (warp >= 17) {
+        // ------------------------------------------------------------------ MMA issuer of query tile t
+        const int t = warp - 17;
+        if (t < nq) {
+            const uint32_t idesc_s = tc::idesc_bf16(BQ, BKV), idesc_o = tc::idesc_bf16(BQ, DP);
+            const uint32_t qa = tc::smem_u32(tiles + G::OFF_Q) + t * G::QK_BYTES, k_base = tc::smem_u32(tiles + G::OFF_K);
+            const uint32_t v_base = tc::smem_u32(tiles + G::OFF_V), pa = tc::smem_u32(tiles + G::OFF_P) + t * G::P_BYTES;
+            const uint32_t d_s = tmem_base + t * 128, d_o = tmem_base + 256 + t * 128;
+            // operand descriptors are fixed per buffer: built once
+            constexpr int KS = DP / 16;
+            uint64_t qd[KS], kd[2][KS], pd[8], vd[2][8];
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-                tc::mma_bf16(d, tc::smem_desc(qa + k * 32, 1024, 2), tc::smem_desc(ka + k * 32, 1024, 2), idesc_s, k != 0);
-#pragma unroll
-            for (int k = 0; k < G::W1 / 16; ++k)
-                tc::mma_bf16(d, tc::smem_desc(qa + G::QK0_BYTES + k * 32, 8 * G::ROW1, G::LAY1),
-                             tc::smem_desc(ka + G::QK0_BYTES + k * 32, 8 * G::ROW1, G::LAY1), idesc_s, 1u);
-            tc::mma_commit(&s_full[t]);
-        };
-        auto issue_o = [&](int t, int vb, uint32_t accumulate) {   // O_t (+)= P_t V over the 128 keys in steps of 16
-            const uint32_t pa = p_base + t * G::P_BYTES, va = v_base + vb * G::V_BYTES, d = tmem_base + 256 + t * 128;
+            for (int k = 0; k < KS; ++k) {
+                if (k < 4) {
+                    qd[k] = tc::smem_desc(qa + k * 32, 1024, 2);
+                    kd[0][k] = tc::smem_desc(k_base + k * 32, 1024, 2);
+                    kd[1][k] = tc::smem_desc(k_base + G::QK_BYTES + k * 32, 1024, 2);
+                } else {
+                    qd[k] = tc::smem_desc(qa + G::QK0_BYTES + (k - 4) * 32, 8 * G::ROW1, G::LAY1);
+                    kd[0][k] = tc::smem_desc(k_base + G::QK0_BYTES + (k - 4) * 32, 8 * G::ROW1, G::LAY1);
+                    kd[1][k] = tc::smem_desc(k_base + G::QK_BYTES + G::QK0_BYTES + (k - 4) * 32, 8 * G::ROW1, G::LAY1);
+                }
+            }
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
                 const uint32_t half = k >> 2, ko = (k & 3) * 32;
-                tc::mma_bf16(d, tc::smem_desc(pa + half * G::P_HALF + ko, 1024, 2),
-                             tc::smem_desc(va + half * G::V_HALF + ko, 1024, 2), idesc_o, (accumulate | (uint32_t)k) != 0 ? 1u : 0u);
+                pd[k] = tc::smem_desc(pa + half * G::P_HALF + ko, 1024, 2);
+                vd[0][k] = tc::smem_desc(v_base + half * G::V_HALF + ko, 1024, 2);
+                vd[1][k] = tc::smem_desc(v_base + G::V_BYTES + half * G::V_HALF + ko, 1024, 2);
             }
-            tc::mma_commit(&o_full[t]);
-        };
-        bool ok = wait(bar_q, 0) && wait(bar_qz, 0) && wait(&k_full[0], 0);
-        if (ok) {
-            tc::tc_fence_after();
-            if (tc::elect_one()) {
-                for (int t = 0; t < nq; ++t) issue_s(t, 0);
-                tc::mma_commit(&k_empty[0]);
-            }
-            __syncwarp();
-        }
-        for (int j = 0; ok && j < nb; ++j) {
-            const int b = j & 1;
-            const uint32_t ph = (uint32_t)j & 1u, bph = (uint32_t)(j >> 1) & 1u;
-            for (int t = 0; ok && t < nq; ++t) {
-                if (j + 1 < nb) {
-                    // S_t of the next block as soon as this tile's softmax has pulled S_t of this block out of TMEM
-                    ok = wait(&s_free[t], ph);
-                    if (ok && t == 0) ok = wait(&k_full[b ^ 1], (uint32_t)((j + 1) >> 1) & 1u);
-                    if (!ok) break;
-                    tc::tc_fence_after();
-                    if (tc::elect_one()) {
-                        issue_s(t, b ^ 1);
-                        if (t == nq - 1) tc::mma_commit(&k_empty[b ^ 1]);
-                    }
-                    __syncwarp();
-                }
-                ok = wait(&p_ready[t], ph);
-                if (ok && t == 0) ok = wait(&v_full[b], bph);
-                if (!ok) break;
+            auto issue_s = [&](int kb) {                        // S_t = Q_t K^T over d_pad in steps of 16 (elected lane)
+#pragma unroll
+                for (int k = 0; k < KS; ++k) tc::mma_bf16(d_s, qd[k], kb ? kd[1][k] : kd[0][k], idesc_s, k != 0);
+                tc::mma_commit(&s_full[t]);
+                tc::mma_commit(&k_empty[kb]);                   // one arrival per tile
+            };
+            auto issue_o = [&](int vb, uint32_t accumulate) {   // O_t (+)= P_t V over the 128 keys in steps of 16
+#pragma unroll
+                for (int k = 0; k < 8; ++k) tc::mma_bf16(d_o, pd[k], vb ? vd[1][k] : vd[0][k], idesc_o, (accumulate | (uint32_t)k) != 0 ? 1u : 0u);
+                tc::mma_commit(&o_full[t]);
+                tc::mma_commit(&v_empty[vb]);
+            };
+            bool ok = wait2(bar_q, 0, bar_qz, 0) && wait(&k_full[0], 0);
+            if (ok) {
                 tc::tc_fence_after();
-                if (tc::elect_one()) {
-                    issue_o(t, b, j > 0 ? 1u : 0u);
-                    if (t == nq - 1) tc::mma_commit(&v_empty[b]);
-                }
+                if (tc::elect_one()) issue_s(0);
                 __syncwarp();
             }
+            for (int j = 0; ok && j < nb; ++j) {
+                const int b = j & 1;
+                const uint32_t ph = (uint32_t)j & 1u, bph = (uint32_t)(j >> 1) & 1u;
+                if (j + 1 < nb) {
+                    // S_t of the next block as soon as this tile's softmax has pulled S_t of this block out of TMEM
+                    ok = wait2(&s_free[t], ph, &k_full[b ^ 1], (uint32_t)((j + 1) >> 1) & 1u);
+                    if (!ok) break;
+                    tc::tc_fence_after();
+                    if (tc::elect_one()) issue_s(b ^ 1);
+                    __syncwarp();
+                }
+                ok = wait2(&p_ready[t], ph, &v_full[b], bph);
+                if (!ok) break;
+                tc::tc_fence_after();
+                if (tc::elect_one()) issue_o(b, j > 0 ? 1u : 0u);
+                __syncwarp();
+            }
+            if (!ok && lane == 0) fail();
         }
-        if (!ok && lane == 0) fail();
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ softmax + output accumulation
-        const int t = warp >> 2, wq = warp & 3;
+        const int t = warp >> 3, hf = (warp >> 2) & 1, wq = warp & 3;
         if (t < nq) {
             const int r = wq * 32 + lane;                          // query row within the tile = TMEM lane
             const uint32_t lane_sel = (uint32_t)(wq * 32) << 16;
-            const uint32_t tmem_S = tmem_base + t * 128 + lane_sel, tmem_O = tmem_base + 256 + t * 128 + lane_sel;
+            const uint32_t tmem_S = tmem_base + t * 128 + hf * 64 + lane_sel, tmem_O = tmem_base + 256 + t * 128 + lane_sel;
             uint8_t* sQ = tiles + G::OFF_Q + t * G::QK_BYTES;
-            uint8_t* prow = tiles + G::OFF_P + t * G::P_BYTES + r * 128;
-            bool ok = wait(bar_q, 0);
-            if (ok) {
-                // zero the Q columns [d_head, d_pad) of this row (they belong to the next head)
-                if constexpr (G::W1 > 0) {
-                    constexpr int units = G::ROW1 / 16, rows_per_128 = 128 / G::ROW1;
-                    for (int u = (a.d_head - 64) / 8; u < units; ++u) {
-                        const int su = u ^ ((r / rows_per_128) & (units - 1));
-                        *reinterpret_cast<uint4*>(sQ + G::QK0_BYTES + r * G::ROW1 + su * 16) = make_uint4(0u, 0u, 0u, 0u);
+            uint8_t* prow = tiles + G::OFF_P + t * G::P_BYTES + hf * G::P_HALF + r * 128;   // this thread's 64 keys of P
+            uint64_t* pbar = &pair_bar[t * 4 + wq];
+            uint32_t xph = 0;                                       // parity of the next row-pair exchange
+            constexpr int NCH = DP / 16;                            // 16-column chunks of O: the two threads of a row split them
+            const int ch0 = hf == 0 ? 0 : (NCH + 1) / 2, ch1 = hf == 0 ? (NCH + 1) / 2 : NCH;
+            bool ok = true;
+            if (hf == 0) {
+                ok = wait(bar_q, 0);
+                if (ok) {
+                    // zero the Q columns [d_head, d_pad) of this row (they belong to the next head)
+                    if constexpr (G::W1 > 0) {
+                        constexpr int units = G::ROW1 / 16, rows_per_128 = 128 / G::ROW1;
+                        for (int u = (a.d_head - 64) / 8; u < units; ++u) {
+                            const int su = u ^ ((r / rows_per_128) & (units - 1));
+                            *reinterpret_cast<uint4*>(sQ + G::QK0_BYTES + r * G::ROW1 + su * 16) = make_uint4(0u, 0u, 0u, 0u);
+                        }
                     }
+                    tc::fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(bar_qz);
                 }
-                tc::fence_proxy_async();
-                __syncwarp();
-                if (lane == 0) tc::mbar_arrive(bar_qz);
             }
-            float m_used = -INFINITY, l_run = 0.f;                  // exponent offset of this row and its running sum
+            float m_used = -INFINITY, l_run = 0.f;                  // exponent offset of this row; sum over this thread's keys
             const float cs = a.scale_log2e;
             for (int j = 0; ok && j < nb; ++j) {
                 const uint32_t ph = (uint32_t)j & 1u;
                 ok = wait(&s_full[t], ph);
                 if (!ok) break;
                 tc::tc_fence_after();
-                uint32_t sv[128];                                   // the whole row of S: one TMEM round trip
-                tc::tmem_ld64(tmem_S, *reinterpret_cast<uint32_t(*)[64]>(&sv[0]));
-                tc::tmem_ld64(tmem_S + 64, *reinterpret_cast<uint32_t(*)[64]>(&sv[64]));
+                uint32_t sv[64];                                    // this thread's half row of S: one TMEM round trip
+                tc::tmem_ld64(tmem_S, sv);
                 tc::tmem_wait_ld();
                 tc::tc_fence_before();
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(&s_free[t]);         // the next block's S may overwrite TMEM now
                 float m0 = __uint_as_float(sv[0]), m1 = __uint_as_float(sv[1]), m2 = __uint_as_float(sv[2]), m3 = __uint_as_float(sv[3]);
 #pragma unroll
-                for (int i = 4; i < 128; i += 4) {
+                for (int i = 4; i < 64; i += 4) {
                     m0 = fmaxf(m0, __uint_as_float(sv[i])); m1 = fmaxf(m1, __uint_as_float(sv[i + 1]));
                     m2 = fmaxf(m2, __uint_as_float(sv[i + 2])); m3 = fmaxf(m3, __uint_as_float(sv[i + 3]));
                 }
-                const float m_new = fmaxf(m_used, fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)));
+                // exchange the half-row maxima with the thread that holds the other 64 keys of this row
+                float* xs = mx_x + ((xph * 2 + t) * 2) * 128;
+                const float m_half = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+                xs[hf * 128 + r] = m_half;
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(pbar);
+                ok = wait(pbar, xph);
+                if (!ok) break;
+                xph ^= 1u;
+                const float m_new = fmaxf(m_used, fmaxf(m_half, xs[(hf ^ 1) * 128 + r]));
                 bool waited_o = false;
                 if (__any_sync(0xffffffffu, (m_new - m_used) * cs > 8.f)) {
-                    // move the exponent offset of the rows of this warp (always on the first block)
+                    // move the exponent offset of the rows of this warp (always on the first block); the partner warp
+                    // takes the same decision from the same values and rescales the other columns of O
                     if (j > 0) {
                         ok = wait(&o_full[t], ph ^ 1u);             // O_t complete up to the previous block
                         if (!ok) break;
                         waited_o = true;
                         tc::tc_fence_after();
                         const float alpha = ex2((m_used - m_new) * cs);
-#pragma unroll
-                        for (int c0 = 0; c0 < DP; c0 += 16) {
+                        for (int ch = ch0; ch < ch1; ++ch) {
                             uint32_t ov[16];
-                            tc::tmem_ld16(tmem_O + c0, ov);
+                            tc::tmem_ld16(tmem_O + ch * 16, ov);
                             tc::tmem_wait_ld();
 #pragma unroll
                             for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
-                            tc::tmem_st16(tmem_O + c0, ov);
+                            tc::tmem_st16(tmem_O + ch * 16, ov);
                         }
                         tc::tmem_wait_st();
                         l_run *= alpha;
@@ -293,7 +329,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
                 const float mc = m_used * cs;
                 float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
-                for (int c0 = 0; c0 < BKV; c0 += 32) {
+                for (int c0 = 0; c0 < 64; c0 += 32) {
                     uint32_t pk[16];
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
@@ -303,11 +339,10 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
                         __nv_bfloat162 bb = __floats2bfloat162_rn(p0, p1);
                         pk[i] = *reinterpret_cast<uint32_t*>(&bb);
                     }
-                    uint8_t* base = prow + (c0 >> 6) * G::P_HALF;
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
-                        const int unit = ((c0 & 63) >> 3) + u;      // 16-byte unit within the 128-byte row
-                        *reinterpret_cast<uint4*>(base + ((unit ^ (r & 7)) << 4)) = make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]);
+                        const int unit = (c0 >> 3) + u;             // 16-byte unit within the 128-byte row
+                        *reinterpret_cast<uint4*>(prow + ((unit ^ (r & 7)) << 4)) = make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]);
                     }
                 }
                 l_run += sum0 + sum1;
@@ -316,14 +351,21 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(&p_ready[t]);
             }
+            // row sum = this thread's keys + the partner's (both were kept at the same exponent offset)
+            if (ok) {
+                l_x[(t * 2 + hf) * 128 + r] = l_run;
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(pbar);
+                ok = wait(pbar, xph);
+            }
             if (ok) ok = wait(&o_full[t], (uint32_t)(nb - 1) & 1u);
             if (ok) {
                 tc::tc_fence_after();
-                const float inv = 1.f / l_run;
+                const float inv = 1.f / (l_run + l_x[(t * 2 + (hf ^ 1)) * 128 + r]);
                 __nv_bfloat16* dst = a.out + ((long long)seq * T + q0 + t * BQ + r) * ((long long)a.heads * a.d_head) + (long long)head * a.d_head;
                 const int dh = a.d_head;                            // multiple of 8
-#pragma unroll
-                for (int c0 = 0; c0 < DP; c0 += 16) {
+                for (int ch = ch0; ch < ch1; ++ch) {
+                    const int c0 = ch * 16;
                     uint32_t ov[16];
                     tc::tmem_ld16(tmem_O + c0, ov);
                     tc::tmem_wait_ld();
@@ -347,7 +389,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
     }
     tc::tc_fence_before();
     __syncthreads();
-    if (warp == 9) { tc::tc_fence_after(); tc::tmem_dealloc(tmem_base, kTmemCols); }
+    if (warp == 17) { tc::tc_fence_after(); tc::tmem_dealloc(tmem_base, kTmemCols); }
 }
 
 template <int DP>
