@@ -13,8 +13,8 @@
 // Per block of 128 keys and per tile, a softmax thread pulls its half row of S out of TMEM in one round trip and
 // releases S at once (the next block's S is issued while this softmax still runs), takes the row maximum, turns the
 // row into exp2 probabilities (row sum in fp32, P rounded to bf16 into shared memory in the MMA operand layout) and
-// signals P; the two threads of a row exchange their half-row maxima through shared memory so that both use the same
-// exponent offset, and add their partial row sums at the end.  O_t accumulates in TMEM across all key blocks: the exponent offset of a row is only moved when the row
+// signals P; the two threads of a row exchange their half-row maxima through shared memory (named barrier of their two
+// warps) so that both use the same exponent offset, and add their partial row sums at the end.  O_t accumulates in TMEM across all key blocks: the exponent offset of a row is only moved when the row
 // maximum has grown by more than 8 (a factor 256), in which case the row's O and running sum are rescaled in place
 // before that block's P V is issued; numerator and denominator always share the offset, so the result is exact.
 // Issue order per block: S_0(next), PV_0, S_1(next), PV_1.
@@ -84,8 +84,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
     uint64_t* p_ready = bar_q + 12;     // [2] per tile: P stored and S consumed (4 warp arrivals)
     uint64_t* o_full = bar_q + 14;      // [2] per tile: O_j complete
     uint64_t* s_free = bar_q + 16;      // [2] per tile: S_j read out of TMEM (4 warp arrivals)
-    uint64_t* pair_bar = bar_q + 18;    // [8] tile * 4 + lane quarter: the two warps that share rows (2 arrivals)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_q + 26);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_q + 18);
     volatile uint32_t* abort_flag = tmem_slot + 1;
     float* mx_x = reinterpret_cast<float*>(smem + 1024);       // [parity][tile][half][row]
     float* l_x = reinterpret_cast<float*>(smem + 5120);        // [tile][half][row]
@@ -100,7 +99,6 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
 
     if (threadIdx.x == 0) {
         tc::mbar_init(bar_q, 1); tc::mbar_init(bar_qz, 4 * nq);
-        for (int i = 0; i < 8; ++i) tc::mbar_init(&pair_bar[i], 2);
         for (int i = 0; i < 2; ++i) {
             tc::mbar_init(&k_full[i], 1); tc::mbar_init(&k_empty[i], nq); tc::mbar_init(&v_full[i], 1); tc::mbar_init(&v_empty[i], nq);
             tc::mbar_init(&s_full[i], 1); tc::mbar_init(&p_ready[i], 8); tc::mbar_init(&o_full[i], 1); tc::mbar_init(&s_free[i], 8);
@@ -249,8 +247,6 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
             const uint32_t tmem_S = tmem_base + t * 128 + hf * 64 + lane_sel, tmem_O = tmem_base + 256 + t * 128 + lane_sel;
             uint8_t* sQ = tiles + G::OFF_Q + t * G::QK_BYTES;
             uint8_t* prow = tiles + G::OFF_P + t * G::P_BYTES + hf * G::P_HALF + r * 128;   // this thread's 64 keys of P
-            uint64_t* pbar = &pair_bar[t * 4 + wq];
-            uint32_t xph = 0;                                       // parity of the next row-pair exchange
             constexpr int NCH = DP / 16;                            // 16-column chunks of O: the two threads of a row split them
             const int ch0 = hf == 0 ? 0 : (NCH + 1) / 2, ch1 = hf == 0 ? (NCH + 1) / 2 : NCH;
             bool ok = true;
@@ -272,92 +268,98 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
             }
             float m_used = -INFINITY, l_run = 0.f;                  // exponent offset of this row; sum over this thread's keys
             const float cs = a.scale_log2e;
-            for (int j = 0; ok && j < nb; ++j) {
+            const int pair_id = 1 + t * 4 + wq;                     // named barrier of the two warps that share these rows
+            auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(pair_id) : "memory"); };
+            // The pair barrier is a hardware barrier (cheap, but unbounded): both warps therefore run it in every
+            // iteration whatever happened before, and a warp whose bounded wait gave up only stops doing work.
+            bool s_polled = false;                                  // an early poll already saw this block's S complete
+            for (int j = 0; j < nb; ++j) {
                 const uint32_t ph = (uint32_t)j & 1u;
-                ok = wait(&s_full[t], ph);
-                if (!ok) break;
-                tc::tc_fence_after();
-                uint32_t sv[64];                                    // this thread's half row of S: one TMEM round trip
-                tc::tmem_ld64(tmem_S, sv);
-                tc::tmem_wait_ld();
-                tc::tc_fence_before();
-                __syncwarp();
-                if (lane == 0) tc::mbar_arrive(&s_free[t]);         // the next block's S may overwrite TMEM now
-                float m0 = __uint_as_float(sv[0]), m1 = __uint_as_float(sv[1]), m2 = __uint_as_float(sv[2]), m3 = __uint_as_float(sv[3]);
+                uint32_t sv[64];                                    // this thread's half row of S
+                float m_half = 0.f;
+                bool o_polled = false;
+                float* xs = mx_x + (((j & 1) * 2 + t) * 2) * 128;
+                if (ok && !s_polled) ok = wait(&s_full[t], ph);
+                if (ok) {
+                    tc::tc_fence_after();
+                    tc::tmem_ld64(tmem_S, sv);                      // one TMEM round trip
+                    tc::tmem_wait_ld();
+                    tc::tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(&s_free[t]);     // the next block's S may overwrite TMEM now
+                    // poll early for the previous P V (its latency hides behind the maximum and the pair barrier)
+                    if (j > 0) o_polled = tc::mbar_try_wait(&o_full[t], ph ^ 1u);
+                    float m0 = __uint_as_float(sv[0]), m1 = __uint_as_float(sv[1]), m2 = __uint_as_float(sv[2]), m3 = __uint_as_float(sv[3]);
 #pragma unroll
-                for (int i = 4; i < 64; i += 4) {
-                    m0 = fmaxf(m0, __uint_as_float(sv[i])); m1 = fmaxf(m1, __uint_as_float(sv[i + 1]));
-                    m2 = fmaxf(m2, __uint_as_float(sv[i + 2])); m3 = fmaxf(m3, __uint_as_float(sv[i + 3]));
+                    for (int i = 4; i < 64; i += 4) {
+                        m0 = fmaxf(m0, __uint_as_float(sv[i])); m1 = fmaxf(m1, __uint_as_float(sv[i + 1]));
+                        m2 = fmaxf(m2, __uint_as_float(sv[i + 2])); m3 = fmaxf(m3, __uint_as_float(sv[i + 3]));
+                    }
+                    m_half = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+                    xs[hf * 128 + r] = m_half;                      // for the thread that holds the other 64 keys of this row
                 }
-                // exchange the half-row maxima with the thread that holds the other 64 keys of this row
-                float* xs = mx_x + ((xph * 2 + t) * 2) * 128;
-                const float m_half = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
-                xs[hf * 128 + r] = m_half;
-                __syncwarp();
-                if (lane == 0) tc::mbar_arrive(pbar);
-                ok = wait(pbar, xph);
-                if (!ok) break;
-                xph ^= 1u;
-                const float m_new = fmaxf(m_used, fmaxf(m_half, xs[(hf ^ 1) * 128 + r]));
-                bool waited_o = false;
-                if (__any_sync(0xffffffffu, (m_new - m_used) * cs > 8.f)) {
-                    // move the exponent offset of the rows of this warp (always on the first block); the partner warp
-                    // takes the same decision from the same values and rescales the other columns of O
-                    if (j > 0) {
-                        ok = wait(&o_full[t], ph ^ 1u);             // O_t complete up to the previous block
-                        if (!ok) break;
-                        waited_o = true;
-                        tc::tc_fence_after();
-                        const float alpha = ex2((m_used - m_new) * cs);
-                        for (int ch = ch0; ch < ch1; ++ch) {
-                            uint32_t ov[16];
-                            tc::tmem_ld16(tmem_O + ch * 16, ov);
-                            tc::tmem_wait_ld();
+                pair_sync();
+                // the previous P V has read P and O_t is complete up to the previous block: P may be overwritten, O rescaled
+                if (ok && j > 0 && !__all_sync(0xffffffffu, o_polled)) ok = wait(&o_full[t], ph ^ 1u);
+                if (ok) {
+                    const float m_new = fmaxf(m_used, fmaxf(m_half, xs[(hf ^ 1) * 128 + r]));
+                    if (__any_sync(0xffffffffu, (m_new - m_used) * cs > 8.f)) {
+                        // move the exponent offset of the rows of this warp (always on the first block); the partner
+                        // warp takes the same decision from the same values and rescales the other columns of O
+                        if (j > 0) {
+                            tc::tc_fence_after();
+                            const float alpha = ex2((m_used - m_new) * cs);
+                            for (int ch = ch0; ch < ch1; ++ch) {
+                                uint32_t ov[16];
+                                tc::tmem_ld16(tmem_O + ch * 16, ov);
+                                tc::tmem_wait_ld();
 #pragma unroll
-                            for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
-                            tc::tmem_st16(tmem_O + ch * 16, ov);
+                                for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+                                tc::tmem_st16(tmem_O + ch * 16, ov);
+                            }
+                            tc::tmem_wait_st();
+                            l_run *= alpha;
                         }
-                        tc::tmem_wait_st();
-                        l_run *= alpha;
+                        m_used = m_new;
                     }
-                    m_used = m_new;
+                    // once, on the first block: tile 1 starts its exponentials when tile 0 has finished its own, so that
+                    // from then on one tile is in its exp2 phase (the unit both tiles share) while the other loads,
+                    // exchanges and stores
+                    if (j == 0 && t == 1) ok = wait(&p_ready[0], 0);
                 }
-                if (j > 0 && !waited_o) {                           // the previous P V has read P: the buffer is free
-                    ok = wait(&o_full[t], ph ^ 1u);
-                    if (!ok) break;
-                }
-                const float mc = m_used * cs;
-                float sum0 = 0.f, sum1 = 0.f;
+                if (ok) {
+                    const float mc = m_used * cs;
+                    float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
-                for (int c0 = 0; c0 < 64; c0 += 32) {
-                    uint32_t pk[16];
+                    for (int c0 = 0; c0 < 64; c0 += 32) {
+                        uint32_t pk[16];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const float p0 = ex2(fmaf(__uint_as_float(sv[c0 + 2 * i]), cs, -mc));
-                        const float p1 = ex2(fmaf(__uint_as_float(sv[c0 + 2 * i + 1]), cs, -mc));
-                        sum0 += p0; sum1 += p1;
-                        __nv_bfloat162 bb = __floats2bfloat162_rn(p0, p1);
-                        pk[i] = *reinterpret_cast<uint32_t*>(&bb);
+                        for (int i = 0; i < 16; ++i) {
+                            const float p0 = ex2(fmaf(__uint_as_float(sv[c0 + 2 * i]), cs, -mc));
+                            const float p1 = ex2(fmaf(__uint_as_float(sv[c0 + 2 * i + 1]), cs, -mc));
+                            sum0 += p0; sum1 += p1;
+                            __nv_bfloat162 bb = __floats2bfloat162_rn(p0, p1);
+                            pk[i] = *reinterpret_cast<uint32_t*>(&bb);
+                        }
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int unit = (c0 >> 3) + u;         // 16-byte unit within the 128-byte row
+                            *reinterpret_cast<uint4*>(prow + ((unit ^ (r & 7)) << 4)) = make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]);
+                        }
                     }
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int unit = (c0 >> 3) + u;             // 16-byte unit within the 128-byte row
-                        *reinterpret_cast<uint4*>(prow + ((unit ^ (r & 7)) << 4)) = make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]);
-                    }
+                    l_run += sum0 + sum1;
+                    // poll early for the next block's S (issued long ago): the answer arrives while P is published
+                    const bool s_next = j + 1 < nb && tc::mbar_try_wait(&s_full[t], ph ^ 1u);
+                    tc::tc_fence_before();
+                    tc::fence_proxy_async();                        // P (generic-proxy stores) visible to the tensor core
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(&p_ready[t]);
+                    s_polled = __all_sync(0xffffffffu, s_next);
                 }
-                l_run += sum0 + sum1;
-                tc::tc_fence_before();
-                tc::fence_proxy_async();                            // P (generic-proxy stores) visible to the tensor core
-                __syncwarp();
-                if (lane == 0) tc::mbar_arrive(&p_ready[t]);
             }
             // row sum = this thread's keys + the partner's (both were kept at the same exponent offset)
-            if (ok) {
-                l_x[(t * 2 + hf) * 128 + r] = l_run;
-                __syncwarp();
-                if (lane == 0) tc::mbar_arrive(pbar);
-                ok = wait(pbar, xph);
-            }
+            l_x[(t * 2 + hf) * 128 + r] = l_run;
+            pair_sync();
             if (ok) ok = wait(&o_full[t], (uint32_t)(nb - 1) & 1u);
             if (ok) {
                 tc::tc_fence_after();
