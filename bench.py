@@ -162,6 +162,23 @@ def make_workload(name, batch, rank):
     raise SystemExit(f"unknown workload {name}")
 
 
+def max_over_ranks(times_ms, device):
+    """Element-wise maximum of per-rank timings over all ranks (every rank gets the result); single process: identity.
+    The job's time is that of its slowest rank."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(t) for t in times_ms]
+    t = torch.tensor(list(times_ms), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_value(units_per_rank_step, world, ms_per_step):
+    """Aggregate throughput of `world` ranks that each process `units_per_rank_step` per step (weak scaling)."""
+    return units_per_rank_step * world / (ms_per_step / 1e3)
+
+
 def cpu_threads():
     try:
         return len(os.sched_getaffinity(0))
@@ -265,13 +282,10 @@ def main():
     barrier()
     ms_e2e = e0.elapsed_time(e1)
 
-    if world > 1:
-        t = torch.tensor([ms, ms_e2e], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = t.tolist()
+    ms, ms_e2e = max_over_ranks([ms, ms_e2e], "cuda")
     ms_step = ms / args.steps
-    value = wl.units_per_step * world / (ms_step / 1e3)
-    e2e_value = wl.units_per_step * world / (ms_e2e / n_e2e / 1e3)
+    value = whole_job_value(wl.units_per_step, world, ms_step)
+    e2e_value = whole_job_value(wl.units_per_step, world, ms_e2e / n_e2e)
 
     if rank == 0:
         out = {"metric": wl.metric, "value": value, "unit": wl.unit, "n_gpus": world, "steps": args.steps,

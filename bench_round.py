@@ -99,16 +99,29 @@ class RoundWorkload:
     def kernel_ms_per_launch(self):
         return None
 
+    # DRAM bytes (read + write) of one fc1 launch at 24 sequences from the ncu capture summarised in
+    # profiles/linear_tc2_kernel_xl_block_24seq.txt; None when the kernel changed after the capture
+    NCU_FC1_DRAM_BYTES_24SEQ = None
+
     def roofline(self, _ms, peaks):
-        """Dominant kernel = the tensor-core linear-layer class with the largest share of device time."""
+        """Dominant kernel = the CTA-pair linear kernel (qkv, proj, fc1, fc2 launches of every pass): algorithmic
+        2 M N K of its launches over their summed device time (CUDA events inside the timed region)."""
         lin = [p for p in self._prof if p["name"].startswith("linear")]
-        top = max(lin, key=lambda p: p["ms"])
-        per_launch_ms = top["ms"] / top["launches"]
-        ach = top["work"] / top["launches"] / 1e12 / (per_launch_ms / 1e3)
+        ms = sum(p["ms"] for p in lin)
+        work = sum(p["work"] for p in lin)
+        launches = sum(p["launches"] for p in lin)
+        ach = work / 1e12 / (ms / 1e3)
         peak = peaks["bf16_tflops_sustained"]
+        top = max(lin, key=lambda p: p["ms"])
+        traffic = None
+        if self.NCU_FC1_DRAM_BYTES_24SEQ is not None:
+            # traffic of the 192-sequence fc1 launch of the packed pass: proportional to M at fixed N, K
+            traffic = self.NCU_FC1_DRAM_BYTES_24SEQ * (self.B * K_DRAFTS * self.G / 24.0)
         return {"bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
-                "traffic": None, "kernel": f"linear_tc_kernel [{top['name']}]", "launches": top["launches"],
-                "ms_per_launch": per_launch_ms, "peak_source": peaks["source"] + " (sustained bf16 GEMM)"}
+                "traffic": traffic, "traffic_of": "fc1 launch of the packed pass (scaled from a 24-sequence ncu capture)",
+                "kernel": "linear_tc2_kernel (qkv, proj, fc1, fc2)", "launches": launches,
+                "ms_per_launch": ms / launches, "largest_class": top["name"],
+                "peak_source": peaks["source"] + " (sustained bf16 GEMM)"}
 
     def extra(self, ms_step, peaks):
         tot = sum(p["ms"] for p in self._prof)
