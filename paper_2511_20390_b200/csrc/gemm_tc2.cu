@@ -38,7 +38,8 @@ constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kABytes = 128 * BK * 2;              // one CTA's A tile of a stage
 constexpr uint32_t kCtrlBytes = 1024;
 constexpr uint32_t kStageBufBytes = 4096;               // 32 rows x 128 bytes
-constexpr uint32_t kStagingBytes = 4 * 2 * kStageBufBytes;
+constexpr int kBufsPerWarp = 4;                         // staging buffers per epilogue warp: stores in flight per warp
+constexpr uint32_t kStagingBytes = 4 * kBufsPerWarp * kStageBufBytes;
 constexpr uint32_t kVBufBytes = 8192;                   // v^T staging: 3 buffers of 4 groups x (8 columns x 128 tokens)
 static_assert(3 * kVBufBytes <= kStagingBytes, "v^T staging must fit");
 constexpr uint32_t kSmemBudget = 227 * 1024;
@@ -133,14 +134,13 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
         // ------------------------------------------------------------------ TMA producer (both CTAs)
         if (lane == 0) { tc::tma_prefetch_desc(&mapA); tc::tma_prefetch_desc(&mapW); }
         const uint32_t full0 = tc::mapa(tc::smem_u32(&full[0]), 0);          // the even CTA's stage barriers
-        uint32_t it = 0;
+        int s = 0;                                           // stage and its phase advance by counting (no divisions in the loop)
+        uint32_t ph = 0;
         bool ok = true;
         for (long long t = first; ok && t < total; t += step) {
             const int m_blk = (int)(t / a.num_n), n_blk = (int)(t % a.num_n);
             const int a_row = m_blk * 256 + (int)rank * 128, w_row = n_blk * BN + (int)rank * (BN / 2);
-            for (int kb = 0; kb < nk; ++kb, ++it) {
-                const int s = it % stages;
-                const uint32_t ph = (it / stages) & 1u;
+            for (int kb = 0; kb < nk; ++kb) {
                 ok = __all_sync(0xffffffffu, !*abort_flag && tc::mbar_wait(&empty[s], ph ^ 1u));
                 if (!ok) { if (lane == 0) fail(FREE_DEV_ERR_EMPTY_WAIT); break; }
                 if (tc::elect_one()) {
@@ -150,6 +150,7 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
                     tc::tma_load_2d_pair(dst + kABytes, &mapW, full0 + 8u * s, kb * BK, w_row);
                 }
                 __syncwarp();
+                if (++s == stages) { s = 0; ph ^= 1u; }
             }
         }
         if (!ok || *abort_flag) {
@@ -162,7 +163,8 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
         // ------------------------------------------------------------------ MMA issuer (even CTA only)
         if (rank == 0) {
             const uint32_t idesc = tc::idesc_bf16(256, BN);
-            uint32_t it = 0, tl = 0;
+            uint32_t tl = 0, ph = 0;
+            int s = 0;
             bool ok = true;
             for (long long t = first; ok && t < total; t += step, ++tl) {
                 const uint32_t acc = tl & 1u, aph = (tl >> 1) & 1u;
@@ -170,9 +172,7 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
                 if (!ok) { if (lane == 0) fail(FREE_DEV_ERR_ACC_EMPTY); break; }
                 tc::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * (uint32_t)BN;
-                for (int kb = 0; kb < nk; ++kb, ++it) {
-                    const int s = it % stages;
-                    const uint32_t ph = (it / stages) & 1u;
+                for (int kb = 0; kb < nk; ++kb) {
                     ok = __all_sync(0xffffffffu, !*abort_flag && tc::mbar_wait(&full[s], ph));
                     if (!ok) { if (lane == 0) fail(FREE_DEV_ERR_FULL_WAIT); break; }
                     tc::tc_fence_after();
@@ -185,6 +185,7 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
                         tc::mma_commit_pair(&empty[s]);      // both CTAs may refill the stage once these MMAs have read it
                     }
                     __syncwarp();
+                    if (++s == stages) { s = 0; ph ^= 1u; }
                 }
                 if (ok && tc::elect_one()) tc::mma_commit_pair(&accf[acc]);   // accumulators complete in both CTAs
                 __syncwarp();
@@ -195,7 +196,7 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
         // ------------------------------------------------------------------ epilogue (both CTAs)
         const int q = warp & 3;                              // TMEM lanes [32q, 32q+32) belong to this warp
         const uint32_t acce0 = tc::mapa(tc::smem_u32(&acce[0]), 0);
-        uint8_t* my_stage = staging + (size_t)q * 2 * kStageBufBytes;
+        uint8_t* my_stage = staging + (size_t)q * kBufsPerWarp * kStageBufBytes;
         constexpr int CH = OUT_BF16 ? 64 : 32;               // columns per staging buffer (128 bytes per row)
         uint32_t tl = 0, nst = 0, eph = 0;
         bool meet_ok = true;
@@ -319,8 +320,8 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
                         }
                     }
                     // stage the 32 x 128-byte block (16-byte units XOR-swizzled by row, as the tensor map expects)
-                    uint8_t* buf = my_stage + (nst & 1u) * kStageBufBytes;
-                    if (lane == 0) tc::bulk_wait_read<1>();              // the store issued from this buffer two chunks ago has read it
+                    uint8_t* buf = my_stage + (nst % kBufsPerWarp) * kStageBufBytes;
+                    if (lane == 0) tc::bulk_wait_read<kBufsPerWarp - 1>();   // the store issued from this buffer kBufsPerWarp chunks ago has read it
                     __syncwarp();
                     uint8_t* rowp = buf + lane * 128;
 #pragma unroll
