@@ -50,7 +50,7 @@ struct Workspace {
     void *temb, *h1, *sc;
     int32_t* lab_seq;
     float *mod, *fmod, *x;
-    void *hn, *qkv, *att, *hmlp, *emb;
+    void *hn, *qkv, *att, *hmlp, *emb, *fin_split;
     float* head_out;
     // sampling loop
     float *x_cur, *m_a, *pack_in, *x_draft, *m_draft, *m_target, *sigma2_bk, *lam_bk, *u_bk;
@@ -88,6 +88,7 @@ Workspace plan(const free_ctx* c, int n, void* base) {
     w.hmlp = take(M * (size_t)c->F * as);
     w.emb = take(M * D * as);
     w.head_out = (float*)take(M * c->out_dim * 4);
+    w.fin_split = take((size_t)c->out_dim * D * 2 * 2);       // bf16 hi and lo planes of the head matrix
     const size_t dl = c->d_latent;
     w.x_cur = (float*)take(n * dl * 4);
     w.m_a = (float*)take(n * dl * 4);
@@ -199,17 +200,36 @@ int run_blocks(const free_ctx* c, const Workspace& w, const Stack& st, int S, cu
     return FREE_OK;
 }
 
-// modulated head: LayerNorm + (shift, scale) in fp32, then the narrow projection on CUDA cores in fp32 (a bf16
-// tensor-core head was measured to raise the error of the noise prediction from 1.1e-2 to 1.4e-2 of the 2e-2 bound
-// on the XL/2 512 test, for 1.3% of the step time: not worth the margin)
+// modulated head: LayerNorm + (shift, scale), then the narrow projection (N = p*p*c_out, 32 for the */2 models).
+// fp32 mode: CUDA cores.  bf16 mode: tensor cores at fp32-level accuracy -- a plain bf16 head was measured to raise
+// the error of the noise prediction from 1.1e-2 to 1.4e-2 of the 2e-2 bound, so activations and weights are each
+// split into bf16 hi + lo planes and  y W^T ~ y_hi W_hi^T + y_lo W_hi^T + y_hi W_lo^T  (the dropped lo*lo term
+// is 2^-16 relative) is accumulated in fp32 by three small GEMMs.
 int run_head(const free_ctx* c, const Workspace& w, const Stack& st, int S, cudaStream_t s) {
     const free_model_desc& m = c->m;
-    const int D = m.D, T = c->n_tok, M = S * T;
-    Scope prof(c, PC_HEAD, 2.0 * M * D * c->out_dim, s);
-    FREE_TRY(ln_modulate(FREE_FP32, M, D, T, w.x, w.fmod, w.fmod + D, 2LL * D, w.hn, s));
+    const int D = m.D, T = c->n_tok, M = S * T, N = c->out_dim;
+    Scope prof(c, PC_HEAD, 2.0 * M * D * N, s);
     LinearArgs a;
-    a.M = M; a.N = c->out_dim; a.K = D; a.A = w.hn; a.W = st.fin_w; a.bias = st.fin_b;
+    a.M = M; a.N = N; a.K = D; a.bias = st.fin_b;
     a.epi = EPI_BIAS; a.out_dtype = FREE_FP32; a.out = w.head_out;
+    if (m.dtype == FREE_BF16 && linear_bf16_supported(N, D)) {
+        void* w_hi = w.fin_split;
+        void* w_lo = (char*)w.fin_split + (size_t)N * D * 2;
+        const void* y_hi = w.hn;
+        const void* y_lo = (const char*)w.hn + (size_t)M * D * 2;
+        FREE_TRY(split_bf16((long long)N * D, st.fin_w, w_hi, w_lo, s));
+        FREE_TRY(ln_modulate_split(M, D, T, w.x, w.fmod, w.fmod + D, 2LL * D, w.hn, s));
+        a.err = w.err;
+        a.A = y_hi; a.W = w_hi;
+        FREE_TRY(linear_bf16(a, s));                              // bias + y_hi W_hi^T
+        a.epi = EPI_GATE_RESIDUAL; a.bias = nullptr; a.out = nullptr; a.resid = w.head_out; a.gate = nullptr; a.rows_per_seq = T;
+        a.A = y_lo; a.W = w_hi;
+        FREE_TRY(linear_bf16(a, s));                              // += y_lo W_hi^T
+        a.A = y_hi; a.W = w_lo;
+        return linear_bf16(a, s);                                 // += y_hi W_lo^T
+    }
+    FREE_TRY(ln_modulate(FREE_FP32, M, D, T, w.x, w.fmod, w.fmod + D, 2LL * D, w.hn, s));
+    a.A = w.hn; a.W = st.fin_w;
     return linear_fp32(a, s);
 }
 

@@ -62,6 +62,10 @@ int patch_embed(int out_dtype, int n_states, int G, int C, int H, int W, int p, 
 int ln_modulate(int out_dtype, int M, int D, int rows_per_seq, const float* x, const float* shift, const float* scale,
                 long long mod_stride, void* y, cudaStream_t s);
 int convert_rows(int out_dtype, long long n, const float* x, void* y, cudaStream_t s);
+// y = modulated LayerNorm as two bf16 planes: hi = bf16(y) at y_split[0 .. M*D), lo = bf16(y - hi) behind it
+int ln_modulate_split(int M, int D, int rows_per_seq, const float* x, const float* shift, const float* scale,
+                      long long mod_stride, void* y_split, cudaStream_t s);
+int split_bf16(long long n, const float* w, void* hi, void* lo, cudaStream_t s);   // hi = bf16(w), lo = bf16(w - hi)
 int head_to_mean(int n_states, int G, int C, int H, int W, int p, int c_out, float cfg_scale, int N_sched,
                  const float* head_out /*[S*n_tok, p*p*c_out]*/, const float* x_in, long long x_stride,
                  const int32_t* t_idx, const float* coef_x, const float* coef_eps, const float* sigma2,

@@ -114,7 +114,9 @@ __global__ void __launch_bounds__(128) patch_embed_generic_kernel(int G, int C, 
 // One warp per row.  VPL > 0: the row (D = 128 * VPL) lives in registers as VPL float4 per lane; warps stride
 // over the rows and issue the loads of their next row before reducing the current one, so that each warp always
 // has a full row of 16-byte loads in flight (the kernel is a pure stream: read 4 D, write 2 D or 4 D bytes per row).
-template <typename T, int VPL>
+// SPLIT (bf16 only): y is written as two bf16 planes, hi = bf16(y) at y[0 .. M D) and lo = bf16(y - hi) at
+// y[M D .. 2 M D), so that a tensor-core product can recover fp32-level accuracy from hi and lo terms.
+template <typename T, int VPL, bool SPLIT = false>
 __global__ void __launch_bounds__(256, 2) ln_modulate_kernel(int M, int D, int rows_per_seq, const float* __restrict__ x,
                                                              const float* __restrict__ shift, const float* __restrict__ scale,
                                                              long long mod_stride, T* __restrict__ y) {
@@ -165,6 +167,13 @@ __global__ void __launch_bounds__(256, 2) ln_modulate_kernel(int M, int D, int r
                     pk.x = *reinterpret_cast<uint32_t*>(&lo);
                     pk.y = *reinterpret_cast<uint32_t*>(&hi);
                     reinterpret_cast<uint2*>(y + (long long)row * D)[i * 32 + lane] = pk;
+                    if (SPLIT) {                                    // residual plane: what bf16 rounding lost
+                        const float2 f01 = __bfloat1622float2(lo), f23 = __bfloat1622float2(hi);
+                        __nv_bfloat162 r01 = __floats2bfloat162_rn(o0 - f01.x, o1 - f01.y), r23 = __floats2bfloat162_rn(o2 - f23.x, o3 - f23.y);
+                        pk.x = *reinterpret_cast<uint32_t*>(&r01);
+                        pk.y = *reinterpret_cast<uint32_t*>(&r23);
+                        reinterpret_cast<uint2*>(y + (long long)M * D + (long long)row * D)[i * 32 + lane] = pk;
+                    }
                 }
             }
         }
@@ -178,9 +187,22 @@ __global__ void __launch_bounds__(256, 2) ln_modulate_kernel(int M, int D, int r
             float q = 0.f;
             for (int c = lane; c < D; c += 32) { float a = xr[c] - mu; q += a * a; }
             const float rstd = rsqrtf(free_warp_sum(q) * invD + 1e-6f);
-            for (int c = lane; c < D; c += 32)
-                store_act(y + (long long)row * D + c, (xr[c] - mu) * rstd * (1.f + scale[mo + c]) + shift[mo + c]);
+            for (int c = lane; c < D; c += 32) {
+                const float o = (xr[c] - mu) * rstd * (1.f + scale[mo + c]) + shift[mo + c];
+                store_act(y + (long long)row * D + c, o);
+                if (SPLIT) store_act(y + (long long)M * D + (long long)row * D + c, o - (float)y[(long long)row * D + c]);
+            }
         }
+    }
+}
+
+// w (fp32) -> hi = bf16(w), lo = bf16(w - hi)
+__global__ void split_bf16_kernel(long long n, const float* __restrict__ w, __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        const float v = w[i];
+        const __nv_bfloat16 h = __float2bfloat16(v);
+        hi[i] = h;
+        lo[i] = __float2bfloat16(v - __bfloat162float(h));
     }
 }
 
@@ -313,6 +335,30 @@ int ln_modulate(int out_dtype, int M, int D, int rows_per_seq, const float* x, c
     if (M < 1 || D < 1 || rows_per_seq < 1 || !x || !shift || !scale || !y) return FREE_ERR_ARG;
     return out_dtype == FREE_FP32 ? ln_launch<float>(M, D, rows_per_seq, x, shift, scale, mod_stride, (float*)y, s)
                                   : ln_launch<__nv_bfloat16>(M, D, rows_per_seq, x, shift, scale, mod_stride, (__nv_bfloat16*)y, s);
+}
+
+// bf16 hi / lo planes of the modulated LayerNorm (hi at y, lo at y + M*D elements)
+int ln_modulate_split(int M, int D, int rows_per_seq, const float* x, const float* shift, const float* scale,
+                      long long mod_stride, void* y, cudaStream_t s) {
+    if (M < 1 || D < 1 || rows_per_seq < 1 || !x || !shift || !scale || !y) return FREE_ERR_ARG;
+    __nv_bfloat16* yb = (__nv_bfloat16*)y;
+    const unsigned need = (unsigned)((M + 7) / 8), cap = 148u * 2u;
+    const unsigned grid = need < cap ? need : cap;
+    const bool vec = (D % 128 == 0) && (mod_stride % 4 == 0) && free_aligned16(shift) && free_aligned16(scale) && free_aligned16(x) &&
+                     free_aligned16(y) && ((long long)M * D) % 8 == 0;
+    const int vpl = vec ? D / 128 : 0;
+    switch (vpl) {
+        case 3: ln_modulate_kernel<__nv_bfloat16, 3, true><<<grid, 256, 0, s>>>(M, D, rows_per_seq, x, shift, scale, mod_stride, yb); break;
+        case 9: ln_modulate_kernel<__nv_bfloat16, 9, true><<<grid, 256, 0, s>>>(M, D, rows_per_seq, x, shift, scale, mod_stride, yb); break;
+        default: ln_modulate_kernel<__nv_bfloat16, 0, true><<<grid, 256, 0, s>>>(M, D, rows_per_seq, x, shift, scale, mod_stride, yb); break;
+    }
+    return free_check_launch();
+}
+
+int split_bf16(long long n, const float* w, void* hi, void* lo, cudaStream_t s) {
+    const unsigned grid = (unsigned)((n + 255) / 256 > 148 * 8 ? 148 * 8 : (n + 255) / 256);
+    split_bf16_kernel<<<grid, 256, 0, s>>>(n, w, (__nv_bfloat16*)hi, (__nv_bfloat16*)lo);
+    return free_check_launch();
 }
 
 int convert_rows(int out_dtype, long long n, const float* x, void* y, cudaStream_t s) {
