@@ -93,3 +93,22 @@ def test_bf16_trajectory_teacher_forced(free):
     # K = 0: plain sampler, N target calls per sample
     xf3, st3 = model.sample_trajectory(cu(x0), labels, dsched, 0, 0.0, cu(zt))
     assert st3["target_calls"] == B * N
+
+
+def test_ragged_row_blocks_and_single_query_tile(free):
+    # 3 sequences of 128 tokens: 384 rows = one and a half 256-row tiles of the CTA-pair GEMM (the second CTA of the
+    # last pair has no rows), and an attention CTA with a single query tile
+    import dataclasses
+    sh = dataclasses.replace(synth.DIT_S2, depth=2, H=16, W=32)
+    w = synth.make_target_weights(sh, 31, bf16=True, ada_std=0.2, out_gain=2.0)
+    model = free.Model(sh, w, None, dtype="bf16")
+    N = 250
+    sc = osched.make("respaced", N)
+    dsched = free.DeviceSchedule(free.respaced_schedule(N))
+    x = synth.normal(9, 1, (3, sh.C, sh.H, sh.W))
+    t, y = np.array([200, 90, 3], np.int32), np.array([5, 77, 999], np.int32)
+    mean, eps, feat = model.dit_verify_pass(cu(x), cu(t, torch.int32), cu(y, torch.int32), 0.0, dsched, want_eps=True, want_feat=True)
+    torch.cuda.synchronize()
+    assert model.device_error() == 0
+    mo, eo, fo = odit.verify_pass(w, sh, sc, x, t, y, 0.0)
+    assert max(nerr(eps, eo), nerr(mean, mo), nerr(feat, fo)) < TOL

@@ -61,3 +61,24 @@ def test_xl_round_consistency(xl):
     torch.cuda.synchronize()
     assert all(a <= 1 for a in n2.tolist()) or True
     assert torch.isfinite(x1).all() and torch.isfinite(x2).all()
+
+
+def test_xl_256_packed_pass_sampled_against_oracle():
+    # DiT-XL/2-shaped at 256^2: 256 tokens, B = 8 samples x K = 6 states, guidance scale 4 (96 sequences in one pass)
+    import paper_2511_20390_b200 as free
+    sh = synth.DIT_XL2_256
+    w = synth.make_target_weights(sh, 13, bf16=True, ada_std=0.1, out_gain=2.0)
+    model = free.Model(sh, w, None, dtype="bf16")
+    N, B, K = 250, 8, 6
+    sc = osched.make("respaced", N)
+    dsched = free.DeviceSchedule(free.respaced_schedule(N))
+    x, t, y = synth.pack_states(19, B, K, (sh.C, sh.H, sh.W), N, sh.n_classes)
+    X, T, Y = x.reshape(B * K, sh.C, sh.H, sh.W), t.reshape(-1), y.reshape(-1)
+    mean, eps, feat = model.dit_verify_pass(cu(X), cu(T, torch.int32), cu(Y, torch.int32), 4.0, dsched, want_eps=True, want_feat=True)
+    torch.cuda.synchronize()
+    assert model.device_error() == 0
+    pick = [0, 41]
+    mo, eo, fo = odit.verify_pass(w, sh, sc, X[pick], T[pick], Y[pick], 4.0)
+    errs = (nerr(eps[pick], eo), nerr(mean[pick], mo), nerr(feat[pick], fo))
+    print("XL/2 256 errors eps/mean/feat:", errs)
+    assert max(errs) < TOL
