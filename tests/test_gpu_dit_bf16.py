@@ -1,5 +1,5 @@
 """bf16 tensor-core mode against the fp64 oracle on bf16-representable weights.
-Tolerance 2e-2 = max error / max |oracle| per output tensor (the bound the task fixes for bf16)."""
+Tolerance 2e-2 = max error / max |oracle| per output tensor (the bound stated for the bf16 mode of this library)."""
 import numpy as np
 import pytest
 import torch
