@@ -241,6 +241,11 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     import paper_2511_20390_b200 as free
     free.lib()        # fail loudly if the CUDA library is not built
+    if args.workload == "trajectory":     # whole trajectories have their own protocol (one step takes tens of seconds)
+        if rank == 0:
+            from bench_round import run_trajectory
+            run_trajectory(args)
+        return
 
     wl = make_workload(args.workload, args.batch, rank)
     peaks = measured_peaks()

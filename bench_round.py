@@ -227,3 +227,50 @@ class OpsWorkload:
     def oracle_sample(self):
         import synth
         return oracle_dit_sample(synth.DIT_XL2_512, 1)
+
+
+def run_trajectory(args):
+    """`bench.py --workload trajectory`: whole sampling trajectories (Algorithm 1 end to end through sample_trajectory)
+    on the DiT-XL/2-shaped 512^2 model, 250 transitions, guidance, batch B: images per second for the two bounding
+    acceptance regimes (u = 0: every draft accepted; u = 1: a draft is accepted only if its log-ratio is >= 0, which a
+    random-init drafter almost never reaches), for seeded uniforms, and for the plain sequential sampler (K = 0) on
+    the same GPU.  One trajectory per regime after one warm-up trajectory; device time by CUDA events."""
+    import json
+    import torch
+    import synth
+    import paper_2511_20390_b200 as free
+    torch.cuda.set_device(0)
+    sh = synth.DIT_XL2_512
+    B = args.batch or 16
+    model = free.Model.random(sh, 1234, dtype="bf16", with_drafter=True)
+    sched = free.DeviceSchedule(free.respaced_schedule(N_SCHED))
+    g = torch.Generator(device="cuda"); g.manual_seed(7)
+    d = sh.d_latent
+    rn = lambda *s_: torch.randn(*s_, generator=g, device="cuda", dtype=torch.float32)
+    x0 = rn(B, sh.C, sh.H, sh.W)
+    labels = torch.randint(0, sh.n_classes, (B,), generator=g, device="cuda", dtype=torch.int32)
+    zt, zd = rn(B, N_SCHED, d), rn(B, N_SCHED, d)
+    regimes = {"all_accepted": (K_DRAFTS, torch.zeros(B, N_SCHED, device="cuda")),
+               "almost_all_rejected": (K_DRAFTS, torch.ones(B, N_SCHED, device="cuda")),
+               "seeded_uniforms": (K_DRAFTS, torch.rand(B, N_SCHED, generator=g, device="cuda")),
+               "sequential_K0": (0, None)}
+    model.sample_trajectory(x0, labels, sched, K_DRAFTS, CFG, zt, zd, regimes["all_accepted"][1])      # warm-up
+    torch.cuda.synchronize()
+    out = {}
+    for name, (K, u) in regimes.items():
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        x, st = model.sample_trajectory(x0, labels, sched, K, CFG, zt, zd if K else None, u)
+        e1.record()
+        torch.cuda.synchronize()
+        sec = e0.elapsed_time(e1) / 1e3
+        assert torch.isfinite(x).all()
+        out[name] = {"images_per_s": B / sec, "seconds": sec, "rounds": st["rounds"], "target_calls": st["target_calls"],
+                     "draft_calls": st["draft_calls"], "accepted": st["accepted"], "rejected": st["rejected"],
+                     "parallel_efficiency": st["parallel_efficiency"]}
+    line = {"metric": "images/s", "value": out["all_accepted"]["images_per_s"], "unit": "images/s", "n_gpus": 1,
+            "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"sample_trajectory, DiT-XL/2-shaped 512^2, {N_SCHED} transitions, K={K_DRAFTS}, cfg {CFG}, batch {B}; "
+                                   "value = the all-accepted regime"},
+            "regimes": out}
+    print(json.dumps(line))
