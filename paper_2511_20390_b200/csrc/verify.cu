@@ -65,6 +65,20 @@ __global__ void __launch_bounds__(kThreads) spec_verify_kernel(VerifyArgs a) {
             const float4* px = reinterpret_cast<const float4*>(a.xh + off);
             const long long n4 = d >> 2;
             long long i = first;
+            for (; i + 3LL * stride < n4; i += 4LL * stride) {   // four independent 16-byte loads per stream in flight
+                float4 m0 = __ldg(pm + i), h0 = __ldg(ph + i), x0 = __ldg(px + i);
+                float4 m1 = __ldg(pm + i + stride), h1 = __ldg(ph + i + stride), x1 = __ldg(px + i + stride);
+                float4 m2 = __ldg(pm + i + 2 * stride), h2 = __ldg(ph + i + 2 * stride), x2 = __ldg(px + i + 2 * stride);
+                float4 m3 = __ldg(pm + i + 3 * stride), h3 = __ldg(ph + i + 3 * stride), x3 = __ldg(px + i + 3 * stride);
+                accumulate(s1, s2, m0.x, h0.x, x0.x); accumulate(s1, s2, m0.y, h0.y, x0.y);
+                accumulate(s1, s2, m0.z, h0.z, x0.z); accumulate(s1, s2, m0.w, h0.w, x0.w);
+                accumulate(s1, s2, m1.x, h1.x, x1.x); accumulate(s1, s2, m1.y, h1.y, x1.y);
+                accumulate(s1, s2, m1.z, h1.z, x1.z); accumulate(s1, s2, m1.w, h1.w, x1.w);
+                accumulate(s1, s2, m2.x, h2.x, x2.x); accumulate(s1, s2, m2.y, h2.y, x2.y);
+                accumulate(s1, s2, m2.z, h2.z, x2.z); accumulate(s1, s2, m2.w, h2.w, x2.w);
+                accumulate(s1, s2, m3.x, h3.x, x3.x); accumulate(s1, s2, m3.y, h3.y, x3.y);
+                accumulate(s1, s2, m3.z, h3.z, x3.z); accumulate(s1, s2, m3.w, h3.w, x3.w);
+            }
             for (; i + stride < n4; i += 2 * stride) {     // two independent 16-byte loads per stream in flight
                 float4 m0 = __ldg(pm + i), h0 = __ldg(ph + i), x0 = __ldg(px + i);
                 float4 m1 = __ldg(pm + i + stride), h1 = __ldg(ph + i + stride), x1 = __ldg(px + i + stride);
