@@ -51,7 +51,8 @@ def _compare(m, mh, xh, s2, u, lam=None, n_valid=None):
 
 @pytest.mark.parametrize("B,K,d,c", [(1, 6, 16384, 0.5), (3, 6, 16384, 1.0), (5, 16, 4096, 0.3), (2, 2, 16384, 50.0),
                                      (7, 8, 1000, 1.0), (4, 4, 1003, 0.7), (3, 64, 256, 0.2), (9, 3, 6, 1.5),
-                                     (2, 5, 2048 + 4, 1.0), (33, 6, 16384, 0.8), (3, 6, 4096 + 1, 1.0)])
+                                     (2, 5, 2048 + 4, 1.0), (33, 6, 16384, 0.8), (3, 6, 4096 + 1, 1.0),
+                                     (100, 6, 16384, 0.8), (300, 2, 8192, 1.0), (4, 33, 16384, 0.5)])
 def test_strict_matches_oracle(B, K, d, c):
     # c = |m_hat - m| / sigma of a typical draft: around 1 gives mixed decisions, 50 rejects at once
     sc = osched.make("respaced", 250)
@@ -76,6 +77,23 @@ def test_mixed_decisions_relaxed_and_ragged():
     nv = (np.arange(B) % (K + 1)).astype(np.int32)
     n_r, _ = _compare(m, mh, xh, s2, u, n_valid=nv)
     assert np.all(n_r <= nv)
+
+
+@pytest.mark.parametrize("K", [2, 4, 6, 8, 16])
+@pytest.mark.parametrize("s_rel", [0.01, 0.1, 1.0])
+def test_sweep_strict_and_relaxed(K, s_rel):
+    # the standalone sweep: d = 4x64x64, draft = target + N(0, s^2) with s relative to the step's sigma, per-step
+    # variances from the 250-step schedule, strict rule and two relaxation levels
+    B, d = 8, 16384
+    sc = osched.make("respaced", 250)
+    s2 = np.tile(sc.sigma2[np.linspace(240, 20, K).astype(int)].astype(np.float32), (B, 1))
+    m, mh, xh, u = synth.verifier_inputs(300 + K, B, K, d, s_rel * float(np.sqrt(s2.mean())) / np.sqrt(d) * 8.0, s2)
+    n_strict, _ = _compare(m, mh, xh, s2, u)
+    prev = n_strict
+    for lam_v in (0.5, 0.1):
+        n_rel, _ = _compare(m, mh, xh, s2, u, lam=np.full((B, K), lam_v, np.float32))
+        assert np.all(n_rel >= prev)                                   # a smaller lambda never rejects earlier
+        prev = n_rel
 
 
 def test_degenerate_cases():
