@@ -12,6 +12,18 @@ torch.set_default_dtype(torch.float64)
 
 
 # ----------------------------------------------------------------------------- schedule
+def _golden():
+    """key -> (value, tolerance) from tests/golden/paper_values.txt (the values the paper prints, each with its citation)."""
+    import os
+    out = {}
+    with open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "paper_values.txt")) as fh:
+        for line in fh:
+            line = line.split("#", 1)[0].split()
+            if len(line) == 3:
+                out[line[0]] = (float(line[1]), float(line[2]))
+    return out
+
+
 @pytest.mark.parametrize("kind,N", [("linear", 50), ("respaced", 250)])
 def test_posterior_variance_is_the_gaussian_posterior(kind, N):
     # beta~ must be the variance of q(x_{t-1} | x_t, x_0): precision = alpha/beta + 1/(1 - abar_prev).
@@ -183,11 +195,13 @@ def test_packed_states_are_independent_sequences():
 # ----------------------------------------------------------------------------- sizes the paper quotes
 def test_sizes_quoted_by_the_paper():
     xl = synth.DIT_XL2_512
-    assert abs(xl.n_params() / 1e6 - 676) < 2.0                      # "676M parameters"
-    assert 28e6 < xl.drafter_params(1) < 33e6                        # "~32M trainable parameters"
-    assert xl.n_tok == 1024 and abs(xl.n_tok * xl.D * 4 / 1e6 - 4.7) < 0.05     # "[1024, 1152] ... ~4.7MB in FP32"
+    g = _golden()
+    assert abs(xl.n_params() / 1e6 - g["target_params_millions"][0]) < g["target_params_millions"][1]
+    assert g["drafter_params_millions_min"][0] * 1e6 < xl.drafter_params(1) < g["drafter_params_millions_max"][0] * 1e6
+    assert xl.n_tok == g["feature_tokens"][0] and xl.D == g["feature_width"][0]
+    assert abs(xl.n_tok * xl.D * 4 / 1e6 - g["feature_megabytes_fp32"][0]) < g["feature_megabytes_fp32"][1]
     ratio = xl.flops_per_sequence(depth=1) / xl.flops_per_sequence()
-    assert np.isclose(ratio, 1 / 28)                                 # one block of 28: "~1/28"
+    assert np.isclose(ratio, 1 / g["drafter_cost_ratio_blocks"][0])
     assert abs(xl.flops_per_sequence() / 1e12 - 1.049) < 0.005
 
 
