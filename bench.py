@@ -130,10 +130,15 @@ class VerifierWorkload:
         self.hv.run()
         return self.hv.h2d_bytes, self.hv.d2h_bytes
 
+    # DRAM bytes (read + write) of one launch at B = 64 from the ncu capture summarised in
+    # profiles/spec_verify_kernel_K16_B64.txt; traffic is proportional to the batch
+    NCU_DRAM_BYTES_B64 = 217.8e6
+
     def roofline(self, ms_per_step, peaks):
         ach = self.bytes_per_step / 1e9 / (ms_per_step / 1e3)
+        traffic = self.NCU_DRAM_BYTES_B64 * self.B / 64.0 if (self.K, self.d) == (16, 16384) else None
         return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": ach / peaks["hbm_gbs"], "traffic": None, "kernel": "spec_verify_kernel",
+                "frac": ach / peaks["hbm_gbs"], "traffic": traffic, "kernel": "spec_verify_kernel",
                 "peak_source": peaks["source"]}
 
     def oracle_sample(self):
