@@ -31,15 +31,15 @@ def test_linear_outputs_stay_in_bounds(M, N, K):
     from paper_2511_20390_b200 import binding as b
     L = b.lib()
     g = torch.Generator(device="cuda"); g.manual_seed(M + N)
-    A = torch.randn(M, K, generator=g, device="cuda").bfloat16()
-    W = (torch.randn(N, K, generator=g, device="cuda") * 0.05).bfloat16()
-    bias = torch.randn(N, generator=g, device="cuda")
-    gate = torch.randn((M + 63) // 64, N, generator=g, device="cuda")
+    A = torch.randn(M, K, generator=g, device="cuda", dtype=torch.float32).bfloat16()
+    W = (torch.randn(N, K, generator=g, device="cuda", dtype=torch.float32) * 0.05).bfloat16()
+    bias = torch.randn(N, generator=g, device="cuda", dtype=torch.float32)
+    gate = torch.randn((M + 63) // 64, N, generator=g, device="cuda", dtype=torch.float32)
     ws = Guarded(256)
     st = torch.cuda.current_stream().cuda_stream
     for epi, od in ((b.EPI_BIAS, b.FREE_BF16), (b.EPI_BIAS, b.FREE_FP32), (b.EPI_BIAS_GELU, b.FREE_BF16), (b.EPI_GATE_RESIDUAL, b.FREE_FP32)):
         out = Guarded(M * N * (2 if od == b.FREE_BF16 else 4))
-        resid = Guarded(M * N * 4, torch.float32, torch.zeros(M * N, device="cuda"))
+        resid = Guarded(M * N * 4, torch.float32, torch.zeros(M * N, device="cuda", dtype=torch.float32))
         ws.t.zero_()
         rc = L.free_op_linear(b.FREE_BF16, epi, od, M, N, K, A.data_ptr(), W.data_ptr(), bias.data_ptr(), out.t.data_ptr(),
                               resid.t.data_ptr(), gate.data_ptr(), gate.stride(0), 64, ws.t.data_ptr(), 256, st)

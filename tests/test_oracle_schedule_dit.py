@@ -8,7 +8,6 @@ import torch.nn.functional as F
 import synth
 from oracle import dit, schedule, drafter
 
-torch.set_default_dtype(torch.float64)
 
 
 # ----------------------------------------------------------------------------- schedule
