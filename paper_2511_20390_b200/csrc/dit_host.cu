@@ -53,7 +53,8 @@ struct Workspace {
     void *hn, *qkv, *att, *hmlp, *emb, *fin_split;
     float* head_out;
     // sampling loop
-    float *x_cur, *m_a, *pack_in, *x_draft, *m_draft, *m_target, *sigma2_bk, *lam_bk, *u_bk;
+    float* fin_bias;
+    float *x_cur, *m_a, *pack_in, *x_draft, *m_draft, *sigma2_bk, *lam_bk, *u_bk, *cx_bk, *ce_bk;
     void *feat0, *feat1;
     int32_t *cur_a, *nv, *n_acc, *t_step, *t_pack, *lab_pack, *t_draft, *act_draft, *active;
     size_t total;
@@ -88,17 +89,19 @@ Workspace plan(const free_ctx* c, int n, void* base) {
     w.hmlp = take(M * (size_t)c->F * as);
     w.emb = take(M * D * as);
     w.head_out = (float*)take(M * c->out_dim * 4);
-    w.fin_split = take((size_t)c->out_dim * D * 2 * 2);       // bf16 hi and lo planes of the head matrix
+    w.fin_split = take((size_t)c->out_dim * D * 2 * 2);       // regrouped head matrix: bf16 hi and lo planes, or one fp32 copy
+    w.fin_bias = (float*)take((size_t)c->out_dim * 4);
     const size_t dl = c->d_latent;
     w.x_cur = (float*)take(n * dl * 4);
     w.m_a = (float*)take(n * dl * 4);
     w.pack_in = (float*)take(n * dl * 4);
     w.x_draft = (float*)take(n * dl * 4);
     w.m_draft = (float*)take(n * dl * 4);
-    w.m_target = (float*)take(n * dl * 4);
     w.sigma2_bk = (float*)take(n * 4);
     w.lam_bk = (float*)take(n * 4);
     w.u_bk = (float*)take(n * 4);
+    w.cx_bk = (float*)take(n * 4);
+    w.ce_bk = (float*)take(n * 4);
     w.feat0 = take(M * D * as);
     w.feat1 = take(M * D * as);
     for (int32_t** p : {&w.cur_a, &w.nv, &w.n_acc, &w.t_step, &w.t_pack, &w.lab_pack, &w.t_draft, &w.act_draft, &w.active})
@@ -205,31 +208,34 @@ int run_blocks(const free_ctx* c, const Workspace& w, const Stack& st, int S, cu
 // the error of the noise prediction from 1.1e-2 to 1.4e-2 of the 2e-2 bound, so activations and weights are each
 // split into bf16 hi + lo planes and  y W^T ~ y_hi W_hi^T + y_lo W_hi^T + y_hi W_lo^T  (the dropped lo*lo term
 // is 2^-16 relative) is accumulated in fp32 by three small GEMMs.
-int run_head(const free_ctx* c, const Workspace& w, const Stack& st, int S, cudaStream_t s) {
+// Output: `out` [S * n_tok, c_out*p*p] with the per-token vector regrouped to (channel, row-in-patch, column-in-patch):
+// the head matrix and bias are copied with their rows in that order first.
+int run_head(const free_ctx* c, const Workspace& w, const Stack& st, int S, float* out, cudaStream_t s) {
     const free_model_desc& m = c->m;
     const int D = m.D, T = c->n_tok, M = S * T, N = c->out_dim;
     Scope prof(c, PC_HEAD, 2.0 * M * D * N, s);
     LinearArgs a;
-    a.M = M; a.N = N; a.K = D; a.bias = st.fin_b;
-    a.epi = EPI_BIAS; a.out_dtype = FREE_FP32; a.out = w.head_out;
+    a.M = M; a.N = N; a.K = D; a.bias = w.fin_bias;
+    a.epi = EPI_BIAS; a.out_dtype = FREE_FP32; a.out = out;
     if (m.dtype == FREE_BF16 && linear_bf16_supported(N, D)) {
         void* w_hi = w.fin_split;
         void* w_lo = (char*)w.fin_split + (size_t)N * D * 2;
         const void* y_hi = w.hn;
         const void* y_lo = (const char*)w.hn + (size_t)M * D * 2;
-        FREE_TRY(split_bf16((long long)N * D, st.fin_w, w_hi, w_lo, s));
+        FREE_TRY(head_weights(true, m.patch, m.c_out, D, st.fin_w, st.fin_b, w_hi, w_lo, w.fin_bias, s));
         FREE_TRY(ln_modulate_split(M, D, T, w.x, w.fmod, w.fmod + D, 2LL * D, w.hn, s));
         a.err = w.err;
         a.A = y_hi; a.W = w_hi;
         FREE_TRY(linear_bf16(a, s));                              // bias + y_hi W_hi^T
-        a.epi = EPI_GATE_RESIDUAL; a.bias = nullptr; a.out = nullptr; a.resid = w.head_out; a.gate = nullptr; a.rows_per_seq = T;
+        a.epi = EPI_GATE_RESIDUAL; a.bias = nullptr; a.out = nullptr; a.resid = out; a.gate = nullptr; a.rows_per_seq = T;
         a.A = y_lo; a.W = w_hi;
         FREE_TRY(linear_bf16(a, s));                              // += y_lo W_hi^T
         a.A = y_hi; a.W = w_lo;
         return linear_bf16(a, s);                                 // += y_hi W_lo^T
     }
+    FREE_TRY(head_weights(false, m.patch, m.c_out, D, st.fin_w, st.fin_b, w.fin_split, nullptr, w.fin_bias, s));
     FREE_TRY(ln_modulate(FREE_FP32, M, D, T, w.x, w.fmod, w.fmod + D, 2LL * D, w.hn, s));
-    a.A = w.hn; a.W = st.fin_w;
+    a.A = w.hn; a.W = w.fin_split;
     return linear_fp32(a, s);
 }
 
@@ -239,6 +245,7 @@ struct PassIO {
     float* mean_out; long long mean_stride;
     float* eps_out;
     void* feat_out;
+    float* head_raw;            // if set: the pass ends with the head's output written here (no guidance, no mean)
     // sampling (optional): sample = mean + sigma * noise
     const float* noise; long long noise_stride;
     float* sample_out; long long sample_stride;
@@ -273,7 +280,8 @@ int target_pass(const free_ctx* c, const Workspace& w, int n_states, float cfg, 
     FREE_TRY(run_blocks(c, w, st, S, s));
     if (io.feat_out) { Scope p(c, PC_EMBED, (double)S * c->n_tok * m.D * 6, s);
                        FREE_TRY(convert_rows(m.dtype, (long long)S * c->n_tok * m.D, w.x, io.feat_out, s)); }
-    FREE_TRY(run_head(c, w, st, S, s));
+    if (io.head_raw) return run_head(c, w, st, S, io.head_raw, s);
+    FREE_TRY(run_head(c, w, st, S, w.head_out, s));
     return tail(c, w, n_states, G, cfg, sch, io, s);
 }
 
@@ -298,7 +306,7 @@ int drafter_pass(const free_ctx* c, const Workspace& w, int n_states, float cfg,
     { const int r2 = lin(c, a, s); delete fc; FREE_TRY(r2); }
     FREE_TRY(run_blocks(c, w, st, S, s));
     if (io.feat_out) { Scope p(c, PC_EMBED, (double)M * D * 6, s); FREE_TRY(convert_rows(m.dtype, (long long)M * D, w.x, io.feat_out, s)); }
-    FREE_TRY(run_head(c, w, st, S, s));
+    FREE_TRY(run_head(c, w, st, S, w.head_out, s));
     return tail(c, w, n_states, G, cfg, sch, io, s);
 }
 
@@ -316,8 +324,9 @@ int check_common(const free_ctx* c, int n_states, const free_schedule* sch, void
 struct RoundArgs {
     int B, K, N;
     const int32_t* labels; const float* sigma2; const float* lambda; const float* uniforms;
+    const float *coef_x, *coef_eps;
     int32_t *cur_a, *nv, *t_step, *t_pack, *lab_pack, *t_draft, *act_draft, *active;
-    float *sigma2_bk, *lam_bk, *u_bk;
+    float *sigma2_bk, *lam_bk, *u_bk, *cx_bk, *ce_bk;
 };
 
 // From the cursors a[b] (next transition, 1-based) derive this round's index tables.
@@ -343,6 +352,8 @@ __global__ void round_setup_kernel(RoundArgs r) {
         r.sigma2_bk[b * K + i] = in ? r.sigma2[s] : 1.f;
         r.lam_bk[b * K + i] = (in && r.lambda) ? r.lambda[t - 1] : 1.f;
         r.u_bk[b * K + i] = in ? r.uniforms[(long long)b * N + (t - 1)] : 0.f;
+        r.cx_bk[b * K + i] = r.coef_x[s];
+        r.ce_bk[b * K + i] = r.coef_eps[s];
     }
 }
 
@@ -469,6 +480,20 @@ extern "C" int dit_verify_pass(free_ctx* c, int n_states, const float* x_in, con
     return target_pass(c, w, n_states, cfg_scale, sch, io, reinterpret_cast<cudaStream_t>(stream));
 }
 
+extern "C" int dit_verify_pass_raw(free_ctx* c, int n_states, const float* x_in, const int32_t* t_idx, const int32_t* labels,
+                                   int guidance, const free_schedule* sch, float* head_out, void* feat_out,
+                                   void* ws, size_t ws_bytes, void* stream) {
+    if (!x_in || !t_idx || !labels || !head_out) return FREE_ERR_ARG;
+    FREE_TRY(check_common(c, n_states, sch, ws, ws_bytes));
+    if (!free_aligned16(x_in) || !free_aligned16(head_out) || !free_aligned16(feat_out)) return FREE_ERR_ALIGN;
+    const Workspace w = plan(c, n_states, ws);
+    FREE_CUDA_TRY(cudaMemsetAsync(w.err, 0, 4, reinterpret_cast<cudaStream_t>(stream)));
+    PassIO io{};
+    io.x_in = x_in; io.x_stride = c->d_latent; io.t_idx = t_idx; io.labels = labels;
+    io.feat_out = feat_out; io.head_raw = head_out;
+    return target_pass(c, w, n_states, guidance ? 2.f : 0.f, sch, io, reinterpret_cast<cudaStream_t>(stream));
+}
+
 extern "C" int draft_step(free_ctx* c, int n_states, const float* x_prev, const void* f_prev, const int32_t* t_idx,
                           const int32_t* labels, float cfg_scale, const free_schedule* sch, const float* noise,
                           float* m_hat, float* x_hat, void* f_next, void* ws, size_t ws_bytes, void* stream) {
@@ -502,8 +527,8 @@ struct RoundIO {
 int one_round(const free_ctx* c, const Workspace& w, const RoundIO& r, cudaStream_t s) {
     const int B = r.B, K = r.K, N = r.sch->N, d = c->d_latent;
     const free_schedule* sch = r.sch;
-    RoundArgs ra{B, K, N, r.labels, sch->sigma2, r.lambda, r.uniforms, w.cur_a, w.nv, w.t_step, w.t_pack, w.lab_pack,
-                 w.t_draft, w.act_draft, w.active, w.sigma2_bk, w.lam_bk, w.u_bk};
+    RoundArgs ra{B, K, N, r.labels, sch->sigma2, r.lambda, r.uniforms, sch->coef_x, sch->coef_eps, w.cur_a, w.nv, w.t_step,
+                 w.t_pack, w.lab_pack, w.t_draft, w.act_draft, w.active, w.sigma2_bk, w.lam_bk, w.u_bk, w.cx_bk, w.ce_bk};
     const unsigned egrid = (unsigned)(((long long)B * d + 255) / 256 > 148 * 8 ? 148 * 8 : ((long long)B * d + 255) / 256);
     { Scope p(c, PC_CTRL, 0, s);
       round_setup_kernel<<<(B + 127) / 128, 128, 0, s>>>(ra);
@@ -533,15 +558,19 @@ int one_round(const free_ctx* c, const Workspace& w, const RoundIO& r, cudaStrea
               FREE_TRY(free_check_launch()); }
             void* tmp = f_prev; f_prev = f_next; f_next = tmp;
         }
-        // (3) one packed target pass over (x_a, x_hat_{a+1..a+K-1}) -> m_{a+1..a+K}
+        // (3) one packed target pass over (x_a, x_hat_{a+1..a+K-1}), stopped at the head's output
         PassIO pi{};
         pi.x_in = w.pack_in; pi.x_stride = d; pi.t_idx = w.t_pack; pi.labels = w.lab_pack;
-        pi.mean_out = w.m_target; pi.mean_stride = d;
+        pi.head_raw = w.head_out;
         FREE_TRY(target_pass(c, w, B * K, r.cfg, sch, pi, s));
-        // (4) sequential verification with the first-rejection break; the finalised state replaces x_cur
-        { Scope p(c, PC_VERIFY, (double)B * (3.0 * K + 1) * d * 4, s);
-          FREE_TRY(spec_verify(B, K, d, w.m_target, w.m_draft, w.x_draft, w.sigma2_bk, w.lam_bk, w.u_bk, w.nv,
-                               w.x_cur, w.n_acc, nullptr, s)); }
+        // (4) guidance, the means m_{a+1..a+K} and the sequential verification with the first-rejection break in one
+        //     kernel; the finalised state replaces x_cur
+        const int G = (r.cfg > 0.f && r.cfg != 1.f) ? 2 : 1;
+        const free_model_desc& m = c->m;
+        { Scope p(c, PC_VERIFY, (double)B * ((2.0 + G) * K + 2) * d * 4, s);
+          FREE_TRY(spec_verify_fused_launch(B, K, m.C, m.H, m.W, m.patch, m.c_out, G, r.cfg, w.head_out, w.pack_in, (long long)K * d,
+                                            w.m_draft, w.x_draft, w.cx_bk, w.ce_bk, w.sigma2_bk, w.lam_bk, w.u_bk, w.nv, 0,
+                                            w.x_cur, w.n_acc, nullptr, nullptr, s)); }
     }
     Scope p(c, PC_CTRL, 0, s);
     cursor_update_kernel<<<(B + 127) / 128, 128, 0, s>>>(B, w.active, w.nv, w.n_acc, w.cur_a);

@@ -65,10 +65,20 @@ int convert_rows(int out_dtype, long long n, const float* x, void* y, cudaStream
 // y = modulated LayerNorm as two bf16 planes: hi = bf16(y) at y_split[0 .. M*D), lo = bf16(y - hi) behind it
 int ln_modulate_split(int M, int D, int rows_per_seq, const float* x, const float* shift, const float* scale,
                       long long mod_stride, void* y_split, cudaStream_t s);
-int split_bf16(long long n, const float* w, void* hi, void* lo, cudaStream_t s);   // hi = bf16(w), lo = bf16(w - hi)
+// head matrix [p*p*c_out, D] and bias with rows regrouped to (channel, row-in-patch, column-in-patch); split: bf16 hi / lo
+// planes into out0 / lo, else an fp32 copy into out0
+int head_weights(bool split, int p, int c_out, int D, const float* w, const float* b, void* out0, void* lo, float* b_out, cudaStream_t s);
 int head_to_mean(int n_states, int G, int C, int H, int W, int p, int c_out, float cfg_scale, int N_sched,
-                 const float* head_out /*[S*n_tok, p*p*c_out]*/, const float* x_in, long long x_stride,
+                 const float* head_out /*[S*n_tok, c_out*p*p], vector order (channel, row, col)*/, const float* x_in, long long x_stride,
                  const int32_t* t_idx, const float* coef_x, const float* coef_eps, const float* sigma2,
                  float* mean_out, long long mean_stride, float* eps_out, long long eps_stride,
                  const float* noise, long long noise_stride, float* sample_out, long long sample_stride,
                  float* sample_out2, long long sample2_stride, const int32_t* sample2_mask, cudaStream_t s);
+
+// ---- verification from the head's output (verify_fused.cu) -------------------------------------
+// As the public spec_verify_fused, with a row stride (elements) for x_first.
+int spec_verify_fused_launch(int B, int K, int C, int H, int W, int patch, int c_out, int G, float cfg_scale,
+                             const float* head_out, const float* x_first, long long x_first_stride,
+                             const float* m_draft, const float* x_draft, const float* coef_x, const float* coef_eps,
+                             const float* sigma2, const float* lambda, const float* u, const int32_t* n_valid, int chunk,
+                             float* x_out, int32_t* n_accept, float* logratio_out, float* means_out, cudaStream_t s);

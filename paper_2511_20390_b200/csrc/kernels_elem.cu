@@ -196,13 +196,26 @@ __global__ void __launch_bounds__(256, 2) ln_modulate_kernel(int M, int D, int r
     }
 }
 
-// w (fp32) -> hi = bf16(w), lo = bf16(w - hi)
-__global__ void split_bf16_kernel(long long n, const float* __restrict__ w, __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+// Head matrix and bias with their rows regrouped from the model's (row-in-patch, column-in-patch, channel) order to
+// (channel, row-in-patch, column-in-patch), so that the C noise channels of a token are one contiguous run of the head's
+// output.  SPLIT: two bf16 planes (hi, lo) for the three-GEMM product; else an fp32 copy.
+template <bool SPLIT>
+__global__ void head_weights_kernel(int p, int c_out, int D, const float* __restrict__ w, const float* __restrict__ b,
+                                    void* __restrict__ out0, __nv_bfloat16* __restrict__ lo, float* __restrict__ b_out) {
+    const long long n = (long long)p * p * c_out * D;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
-        const float v = w[i];
-        const __nv_bfloat16 h = __float2bfloat16(v);
-        hi[i] = h;
-        lo[i] = __float2bfloat16(v - __bfloat162float(h));
+        const int row = (int)(i / D), col = (int)(i % D);
+        const int ch = row / (p * p), pix = row % (p * p);
+        const int src = pix * c_out + ch;
+        const float v = w[(long long)src * D + col];
+        if (SPLIT) {
+            const __nv_bfloat16 h = __float2bfloat16(v);
+            reinterpret_cast<__nv_bfloat16*>(out0)[i] = h;
+            lo[i] = __float2bfloat16(v - __bfloat162float(h));
+        } else {
+            reinterpret_cast<float*>(out0)[i] = v;
+        }
+        if (col == 0) b_out[row] = b ? b[src] : 0.f;
     }
 }
 
@@ -253,7 +266,7 @@ __global__ void __launch_bounds__(256) head_to_mean_kernel(TailArgs a) {
         const int st = (int)(i / d), e = (int)(i % d);
         const int c = e / (a.H * a.W), yy = (e / a.W) % a.H, xx = e % a.W;
         const int tok = (yy / a.p) * gw + xx / a.p;
-        const int vec = ((yy % a.p) * a.p + xx % a.p) * a.c_out + c;
+        const int vec = (c * a.p + yy % a.p) * a.p + xx % a.p;
         float eps = a.head_out[((long long)(st * a.G) * n_tok + tok) * od + vec];
         if (a.G == 2) {
             const float eu = a.head_out[((long long)(st * a.G + 1) * n_tok + tok) * od + vec];
@@ -355,9 +368,11 @@ int ln_modulate_split(int M, int D, int rows_per_seq, const float* x, const floa
     return free_check_launch();
 }
 
-int split_bf16(long long n, const float* w, void* hi, void* lo, cudaStream_t s) {
+int head_weights(bool split, int p, int c_out, int D, const float* w, const float* b, void* out0, void* lo, float* b_out, cudaStream_t s) {
+    const long long n = (long long)p * p * c_out * D;
     const unsigned grid = (unsigned)((n + 255) / 256 > 148 * 8 ? 148 * 8 : (n + 255) / 256);
-    split_bf16_kernel<<<grid, 256, 0, s>>>(n, w, (__nv_bfloat16*)hi, (__nv_bfloat16*)lo);
+    if (split) head_weights_kernel<true><<<grid, 256, 0, s>>>(p, c_out, D, w, b, out0, (__nv_bfloat16*)lo, b_out);
+    else head_weights_kernel<false><<<grid, 256, 0, s>>>(p, c_out, D, w, b, out0, nullptr, b_out);
     return free_check_launch();
 }
 
