@@ -1,6 +1,6 @@
 """Benchmark of the packed parallel-verification path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload round|verifier] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload round|verifier|verifier_fused|trajectory] [--impl reference]
 
 One JSON line on stdout (rank 0).  A "step" is one pass of the hot path over one batch of synthetic
 input resident in HBM; `e2e` repeats it from pinned HOST buffers with the copies inside the timed
@@ -29,6 +29,7 @@ def parse():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--workload", default="default")
     ap.add_argument("--batch", type=int, default=0, help="images per step (0 = workload default)")
+    ap.add_argument("--chunk", type=int, default=0, help="verifier_fused: drafts per early-exit chunk (0 = off)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
@@ -152,9 +153,95 @@ class VerifierWorkload:
         return by / 1e9 / dt, f"{nb} of {self.B} samples of the same batch, full K"
 
 
-def make_workload(name, batch, rank):
+class FusedVerifierWorkload:
+    """Verification from the noise predictions of the packed pass (guidance + Eq. ddpm_update + Algorithm 2 in one
+    kernel) at the same point of the sweep: 4x64x64 latents, two guidance streams, K = 16, B = 256.
+    Inputs (1.1 GB) exceed L2.  Draft means sit about 1.8 sigma from the target means (mixed decisions)."""
+    name = "fused verifier K=16 B=256 latent 4x64x64 guidance"
+    metric, unit, dtype = "verifier HBM GB/s", "GB/s", "f32"
+    shape, G, cfg = (4, 64, 64), 2, 4.0
+
+    def __init__(self, batch, rank, chunk=0):
+        import torch
+        import synth
+        import paper_2511_20390_b200 as free
+        self.torch, self.free = torch, free
+        self.B, self.K, self.d, self.chunk = (batch or 256), 16, int(np.prod(self.shape)), chunk
+        B, K, d = self.B, self.K, self.d
+        sched = free.respaced_schedule(250)
+        s2 = np.tile(sched["sigma2"][np.linspace(240, 20, K).astype(int)].astype(np.float32), (B, 1))
+        sig, ce = float(np.sqrt(s2.mean())), 0.05
+        s = 0.35 * sig / np.sqrt(d)
+        eps, x_first, mh, xh, u = synth.eps_verifier_inputs(2000 + rank, B, K, self.G, self.shape, s, s2, eps_std=s / ce)
+        cx = np.ones((B, K), np.float32)
+        self.host = dict(eps=eps, x_first=x_first, m_hat=mh, x_hat=xh, cx=cx, ce=np.full((B, K), ce, np.float32), sigma2=s2, u=u)
+        self.dev = {k: torch.from_numpy(v).cuda() for k, v in self.host.items()}
+        self.x_out = torch.empty((B,) + self.shape, device="cuda")
+        self.n_acc = torch.empty(B, dtype=torch.int32, device="cuda")
+        self.pinned = None
+        # algorithmic bytes per sample: per draft the noise predictions of both streams, m_hat and x_hat once; the first
+        # state and the output once; the [B,K] scalars
+        self.bytes_per_step = B * (K * (self.G + 2) * d * 4 + 2 * d * 4 + 20 * K)
+        self.units_per_step = self.bytes_per_step / 1e9
+        self.launches_per_step = 1
+        self.config = {"workload": self.name, "B": B, "K": K, "d": d, "chunk": chunk,
+                       "cache": "inputs larger than L2 (1.1 GB per step)"}
+
+    def _call(self, d):
+        self.free.spec_verify_fused(d["eps"], d["x_first"], d["m_hat"], d["x_hat"], d["cx"], d["ce"], d["sigma2"], d["u"],
+                                    self.cfg, chunk=self.chunk, x_out=self.x_out, n_accept=self.n_acc)
+
+    def step(self):
+        self._call(self.dev)
+
+    def host_step(self):
+        torch = self.torch
+        if self.pinned is None:
+            self.pinned = {k: torch.from_numpy(v).pin_memory() for k, v in self.host.items()}
+            self.stage = {k: torch.empty_like(v, device="cuda") for k, v in self.pinned.items()}
+            self.h_x, self.h_n = torch.empty(self.x_out.shape, pin_memory=True), torch.empty(self.B, dtype=torch.int32, pin_memory=True)
+        for k, v in self.pinned.items():
+            self.stage[k].copy_(v, non_blocking=True)
+        self._call(self.stage)
+        self.h_x.copy_(self.x_out, non_blocking=True)
+        self.h_n.copy_(self.n_acc, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        return (sum(v.numel() * v.element_size() for v in self.pinned.values()),
+                self.h_x.numel() * 4 + self.h_n.numel() * 4)
+
+    def bytes_examined(self):
+        """With the early exit only whole chunks up to the first rejection are read: the bytes of those rows."""
+        if self.chunk <= 0:
+            return self.bytes_per_step
+        n = self.n_acc.cpu().numpy().astype(np.int64)
+        rows = np.minimum(self.K, (np.minimum(n, self.K - 1) // self.chunk + 1) * self.chunk)
+        return int((rows * (self.G + 2) * self.d * 4 + 2 * self.d * 4 + 20 * rows).sum())
+
+    def roofline(self, ms_per_step, peaks):
+        ach = self.bytes_examined() / 1e9 / (ms_per_step / 1e3)
+        return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": ach / peaks["hbm_gbs"], "traffic": None, "kernel": "spec_verify_fused_kernel",
+                "peak_source": peaks["source"]}
+
+    def extra(self, ms_step, peaks):
+        return {"accepted_per_sample": float(self.n_acc.float().mean().item()),
+                "bytes_read_fraction": self.bytes_examined() / self.bytes_per_step}
+
+    def oracle_sample(self):
+        from oracle import verify as ov
+        nb, h = 2, self.host
+        t0 = time.perf_counter()
+        ov.spec_verify_from_eps(h["eps"][:nb], h["x_first"][:nb], h["m_hat"][:nb], h["x_hat"][:nb], h["cx"][:nb], h["ce"][:nb],
+                                self.cfg, h["sigma2"][:nb], h["u"][:nb])
+        dt = time.perf_counter() - t0
+        return nb * self.bytes_per_step / self.B / 1e9 / dt, f"{nb} of {self.B} samples of the same batch, full K"
+
+
+def make_workload(name, batch, rank, chunk=0):
     if name in ("verifier",):
         return VerifierWorkload(batch, rank)
+    if name == "verifier_fused":
+        return FusedVerifierWorkload(batch, rank, chunk)
     if name in ("default", "round"):
         try:
             from bench_round import RoundWorkload        # the full packed-verify round (DiT + verifier)
@@ -252,7 +339,7 @@ def main():
             run_trajectory(args)
         return
 
-    wl = make_workload(args.workload, args.batch, rank)
+    wl = make_workload(args.workload, args.batch, rank, args.chunk)
     peaks = measured_peaks()
 
     def barrier():

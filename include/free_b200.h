@@ -135,14 +135,14 @@ int dit_verify_pass(free_ctx* ctx, int n_states,
  * dit_verify_pass_raw -- the packed target pass stopped at the network's output: no guidance, no mean.  Feeds
  * spec_verify_fused(), which applies guidance and Eq. ddpm_update itself (Alg. 1, parallel-means line + verification).
  *   guidance  0: one sequence per state (G = 1); non-zero: conditional and unconditional sequences (G = 2)
- *   head_out  DEVICE fp32 [n_states, G, n_tok, c_out*p*p]: per token one vector ordered (channel, row-in-patch,
- *             column-in-patch) -- the C noise channels of a token are its first C*p*p floats; tokens row-major over
- *             the patch grid; conditional stream first
+ *   eps_out   DEVICE fp32 [n_states, G, C, H, W]: the noise prediction of every stream as an image (the head's first C
+ *             output channels, un-patchified by the head GEMM's own epilogue; the variance channels are not stored);
+ *             conditional stream first
  *   other arguments and errors as for dit_verify_pass.
  */
 int dit_verify_pass_raw(free_ctx* ctx, int n_states,
                         const float* x_in, const int32_t* t_idx, const int32_t* labels, int guidance,
-                        const free_schedule* sched, float* head_out, void* feat_out,
+                        const free_schedule* sched, float* eps_out, void* feat_out,
                         void* ws, size_t ws_bytes, void* stream);
 
 /*
@@ -172,15 +172,15 @@ int spec_verify(int B, int K, int64_t d,
                      float* x_out, int32_t* n_accept, float* logratio_out, void* stream);
 
 /*
- * spec_verify_fused -- spec_verify() fed by the head output of the packed pass instead of by means: per draft k of
- * sample b the kernel forms eps = eps_u + w (eps_c - eps_u) (first C channels; eps = eps_c when G = 1), the target mean
+ * spec_verify_fused -- spec_verify() fed by the noise predictions of the packed pass instead of by means: per draft k
+ * of sample b the kernel forms eps = eps_u + w (eps_c - eps_u) (eps = eps_c when G = 1) and the target mean
  * m_k = coef_x[b,k] x_k - coef_eps[b,k] eps (Eq. ddpm_update) in fp64 registers, and then proceeds exactly as
  * spec_verify.  The packed state x_k is x_first[b] for k = 0 and the previous draft x_draft[b,k-1] after that (Alg. 1:
- * the pass sees the current state and the first K-1 drafts), so the drafts are read once for both roles and the
+ * the pass sees the current state and the first K-1 drafts), so the drafts are fetched once for both roles and the
  * [B,K,d] tensor of target means is never written or read.
- *   C, H, W, patch, c_out   latent geometry and head channels (c_out >= C; H, W multiples of patch); d = C*H*W
- *   G, cfg_scale            streams per state (1 or 2) and the guidance scale w (used when G = 2)
- *   head_out   DEVICE fp32 [B, K, G, n_tok, c_out*p*p], layout of dit_verify_pass_raw
+ *   B, K, d    samples, drafts per sample (1..FREE_MAX_K), elements per state
+ *   G, cfg_scale   streams per state (1 or 2) and the guidance scale w (used when G = 2)
+ *   eps        DEVICE fp32 [B, K, G, d], layout of dit_verify_pass_raw
  *   x_first    DEVICE fp32 [B, d]
  *   m_draft, x_draft        DEVICE fp32 [B, K, d]
  *   coef_x, coef_eps, sigma2, u   DEVICE fp32 [B, K]; lambda DEVICE fp32 [B, K] or NULL; n_valid DEVICE int32 [B] or NULL
@@ -192,8 +192,8 @@ int spec_verify(int B, int K, int64_t d,
  *   means_out  DEVICE fp32 [B, K, d] or NULL: the target means of the examined drafts, rounded to fp32 (diagnostic)
  * No workspace.  Errors: ARG (null pointer, G not 1 or 2), SHAPE, ALIGN, CUDA.
  */
-int spec_verify_fused(int B, int K, int C, int H, int W, int patch, int c_out, int G, float cfg_scale,
-                      const float* head_out, const float* x_first, const float* m_draft, const float* x_draft,
+int spec_verify_fused(int B, int K, int64_t d, int G, float cfg_scale,
+                      const float* eps, const float* x_first, const float* m_draft, const float* x_draft,
                       const float* coef_x, const float* coef_eps, const float* sigma2, const float* lambda,
                       const float* u, const int32_t* n_valid, int chunk,
                       float* x_out, int32_t* n_accept, float* logratio_out, float* means_out, void* stream);
@@ -256,7 +256,7 @@ int sample_trajectory(free_ctx* ctx, int B,
  * spec_round -- the body of Algorithm 1's loop, once: for every sample b whose cursor[b] <= N (cursor = index of
  * the next transition, 1-based), target step on x_cur[b], K drafter steps, packed target pass, verification;
  * x_next[b] is the last finalised state and cursor_next[b] points past it.  sample_trajectory is this call
- * repeated until every cursor exceeds N.  The packed pass ends at the head's output and spec_verify_fused() does the rest.
+ * repeated until every cursor exceeds N.  The packed pass ends at the noise predictions and spec_verify_fused() does the rest.
  * Asynchronous.  Arguments as for sample_trajectory;
  *   x_cur, x_next DEVICE fp32 [B, C, H, W] (may alias); cursor, cursor_next DEVICE int32 [B] (may alias);
  *   n_accept DEVICE int32 [B] or NULL: drafts accepted this round (undefined for samples that drafted nothing).

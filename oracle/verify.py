@@ -79,40 +79,32 @@ def spec_verify(m, m_hat, x_hat, sigma2, u, lam=None, n_valid=None):
     return x_out, n_accept, ell
 
 
-def means_from_head_output(head_tok, x_first, x_hat, coef_x, coef_eps, cfg_scale, C, H, W, patch):
-    """Target means m_1..m_K of one sample from the raw head output of its packed pass (Alg. 1,
+def means_from_stream_eps(eps, x_first, x_hat, coef_x, coef_eps, cfg_scale):
+    """Target means m_1..m_K of one sample from the noise predictions of its packed pass (Alg. 1,
     parallel-means line), so that verification can start from the network output itself.
 
-    head_tok [K, G, n_tok, c_out*p*p]: per token a vector ordered (channel, row-in-patch,
-    column-in-patch), tokens row-major over the patch grid; G = 2 streams (conditional, then
-    unconditional) under guidance, else 1.  Packed state k is x_first for k = 0 and the draft
+    eps [K, G, ...]: per packed state the prediction of G = 2 streams (conditional, then
+    unconditional) under guidance, else of one.  Packed state k is x_first for k = 0 and the draft
     x_hat[k-1] after that (the pass sees the current state and the first K-1 drafts).
-    eps = eps_u + w (eps_c - eps_u) on the first C channels (w = cfg_scale);
-    m_k = coef_x[k] x_k - coef_eps[k] eps_k  (Eq. ddpm_update).  Returns [K, C, H, W]."""
-    head_tok = np.asarray(head_tok, np.float64)
-    K, G = head_tok.shape[:2]
-    p, gh, gw = patch, H // patch, W // patch
-    c_out = head_tok.shape[3] // (p * p)
-    x_hat = np.asarray(x_hat, np.float64).reshape(K, C, H, W)
-    means = np.zeros((K, C, H, W))
+    eps_k = eps_u + w (eps_c - eps_u) with w = cfg_scale (the single stream when G = 1);
+    m_k = coef_x[k] x_k - coef_eps[k] eps_k  (Eq. ddpm_update).  Returns [K, ...]."""
+    eps = np.asarray(eps, np.float64)
+    K, G = eps.shape[:2]
+    x_hat = np.asarray(x_hat, np.float64)
+    means = np.zeros_like(x_hat)
     for k in range(K):
-        img = head_tok[k].reshape(G, gh, gw, c_out, p, p)              # [g, token row, token col, channel, pr, pc]
-        img = img.transpose(0, 3, 1, 4, 2, 5).reshape(G, c_out, H, W)[:, :C]
-        eps = img[0] if G == 1 else img[1] + cfg_scale * (img[0] - img[1])
-        x_k = np.asarray(x_first, np.float64).reshape(C, H, W) if k == 0 else x_hat[k - 1]
-        means[k] = coef_x[k] * x_k - coef_eps[k] * eps
+        e = eps[k, 0] if G == 1 else eps[k, 1] + cfg_scale * (eps[k, 0] - eps[k, 1])
+        x_k = np.asarray(x_first, np.float64) if k == 0 else x_hat[k - 1]
+        means[k] = coef_x[k] * x_k - coef_eps[k] * e
     return means
 
 
-def spec_verify_from_head(head_tok, x_first, m_hat, x_hat, coef_x, coef_eps, cfg_scale, shape4, sigma2, u,
-                          lam=None, n_valid=None):
-    """means_from_head_output for every sample, then the sequential verification loop.
-    head_tok [B,K,G,n_tok,c_out*p*p]; x_first [B,C,H,W]; m_hat, x_hat [B,K,C,H,W]; coef_x, coef_eps,
-    sigma2, u, lam [B,K]; shape4 = (C, H, W, patch).  Returns (x_out, n_accept, ell, means)."""
-    C, H, W, p = shape4
-    B = len(head_tok)
-    means = np.stack([means_from_head_output(head_tok[b], x_first[b], x_hat[b], coef_x[b], coef_eps[b], cfg_scale,
-                                             C, H, W, p) for b in range(B)])
-    x_out, n_accept, ell = spec_verify(means, np.asarray(m_hat, np.float64).reshape(means.shape),
-                                       np.asarray(x_hat, np.float64).reshape(means.shape), sigma2, u, lam, n_valid)
+def spec_verify_from_eps(eps, x_first, m_hat, x_hat, coef_x, coef_eps, cfg_scale, sigma2, u, lam=None, n_valid=None):
+    """means_from_stream_eps for every sample, then the sequential verification loop.
+    eps [B,K,G,...]; x_first [B,...]; m_hat, x_hat [B,K,...]; coef_x, coef_eps, sigma2, u, lam [B,K].
+    Returns (x_out, n_accept, ell, means)."""
+    B = len(eps)
+    means = np.stack([means_from_stream_eps(eps[b], x_first[b], x_hat[b], coef_x[b], coef_eps[b], cfg_scale)
+                      for b in range(B)])
+    x_out, n_accept, ell = spec_verify(means, m_hat, x_hat, sigma2, u, lam, n_valid)
     return x_out, n_accept, ell, means

@@ -72,7 +72,7 @@ _SIGNATURES = {
     "dit_verify_pass_raw": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                                       C.POINTER(ScheduleDesc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "spec_verify": (C.c_int, [C.c_int, C.c_int, C.c_int64] + [C.c_void_p] * 11),
-    "spec_verify_fused": (C.c_int, [C.c_int] * 8 + [C.c_float] + [C.c_void_p] * 10 + [C.c_int] + [C.c_void_p] * 5),
+    "spec_verify_fused": (C.c_int, [C.c_int, C.c_int, C.c_int64, C.c_int, C.c_float] + [C.c_void_p] * 10 + [C.c_int] + [C.c_void_p] * 5),
     "draft_step": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
                              C.POINTER(ScheduleDesc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                              C.c_void_p, C.c_size_t, C.c_void_p]),
@@ -153,24 +153,23 @@ def spec_verify(m, m_hat, x_hat, sigma2, u, lam=None, n_valid=None, want_lograti
     return (x_out, n_accept, ell) if want_logratio else (x_out, n_accept)
 
 
-def spec_verify_fused(head_out, x_first, m_hat, x_hat, coef_x, coef_eps, sigma2, u, cfg_scale, geometry, lam=None,
+def spec_verify_fused(eps, x_first, m_hat, x_hat, coef_x, coef_eps, sigma2, u, cfg_scale, lam=None,
                       n_valid=None, chunk=0, want_logratio=False, want_means=False, x_out=None, n_accept=None):
-    """Verification straight from the packed pass's head output (guidance, Eq. ddpm_update and Algorithm 2 in one
-    kernel).  head_out: CUDA fp32 [B,K,G,n_tok,c_out*p*p]; x_first [B,C,H,W]; m_hat, x_hat [B,K,C,H,W];
-    coef_x, coef_eps, sigma2, u, lam: [B,K]; geometry = (C, H, W, patch, c_out); chunk > 0 enables the early exit.
-    Returns (x_out, n_accept[, ell][, means])."""
-    B, K, G = head_out.shape[:3]
-    Cc, H, W, patch, c_out = (int(v) for v in geometry)
-    for t in (head_out, x_first, m_hat, x_hat, coef_x, coef_eps, sigma2, u):
+    """Verification straight from the packed pass's noise predictions (guidance, Eq. ddpm_update and Algorithm 2 in
+    one kernel).  eps: CUDA fp32 [B,K,G,d...]; x_first [B,d...]; m_hat, x_hat [B,K,d...]; coef_x, coef_eps, sigma2, u,
+    lam: [B,K]; chunk > 0 enables the early exit.  Returns (x_out, n_accept[, ell][, means])."""
+    B, K, G = eps.shape[:3]
+    d = int(np.prod(eps.shape[3:]))
+    for t in (eps, x_first, m_hat, x_hat, coef_x, coef_eps, sigma2, u):
         _dev(t, torch.float32)
-    dev = head_out.device
+    dev = eps.device
     if x_out is None:
-        x_out = torch.zeros((B, Cc, H, W), dtype=torch.float32, device=dev)
+        x_out = torch.zeros((B,) + tuple(eps.shape[3:]), dtype=torch.float32, device=dev)
     if n_accept is None:
         n_accept = torch.empty(B, dtype=torch.int32, device=dev)
     ell = torch.empty((B, K), dtype=torch.float32, device=dev) if want_logratio else None
-    means = torch.zeros((B, K, Cc, H, W), dtype=torch.float32, device=dev) if want_means else None
-    code = lib().spec_verify_fused(B, K, Cc, H, W, patch, c_out, G, float(cfg_scale), _ptr(head_out), _ptr(x_first),
+    means = torch.zeros((B, K) + tuple(eps.shape[3:]), dtype=torch.float32, device=dev) if want_means else None
+    code = lib().spec_verify_fused(B, K, d, G, float(cfg_scale), _ptr(eps), _ptr(x_first),
                                    _ptr(m_hat), _ptr(x_hat), _ptr(coef_x), _ptr(coef_eps), _ptr(sigma2),
                                    _ptr(None if lam is None else _dev(lam, torch.float32)), _ptr(u),
                                    _ptr(None if n_valid is None else _dev(n_valid, torch.int32)), int(chunk),
@@ -390,11 +389,11 @@ class Model:
         return out if len(out) > 1 else mean
 
     def dit_verify_pass_raw(self, x, t_idx, labels, guidance: bool, sched: DeviceSchedule, want_feat=False):
-        """The packed target pass stopped at the head: returns head_out [n, G, n_tok, c_out*p*p] (+ feat)."""
+        """The packed target pass stopped at the network output: returns eps [n, G, C, H, W] (+ feat)."""
         sh = self.shape
         n, G = x.shape[0], 2 if guidance else 1
         _dev(x, torch.float32); _dev(t_idx, torch.int32); _dev(labels, torch.int32)
-        head = torch.empty((n, G, sh.n_tok, sh.c_out * sh.patch * sh.patch), dtype=torch.float32, device=x.device)
+        head = torch.empty((n, G, sh.C, sh.H, sh.W), dtype=torch.float32, device=x.device)
         feat = torch.empty((n, G, sh.n_tok, sh.D), dtype=self.act, device=x.device) if want_feat else None
         ws = self.workspace(n)
         _check(lib().dit_verify_pass_raw(self.ctx, n, _ptr(x), _ptr(t_idx), _ptr(labels), int(bool(guidance)),

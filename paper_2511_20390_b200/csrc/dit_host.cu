@@ -10,7 +10,8 @@ enum { PC_COND = 0, PC_EMBED, PC_LN, PC_QKV, PC_ATTN, PC_PROJ, PC_FC1, PC_FC2, P
 static const char* const kProfNames[PC_N] = {
     "conditioning + modulation tables", "patch embed / feature copy", "layernorm + modulate", "linear qkv",
     "attention", "linear proj (gate + residual)", "linear fc1 + gelu", "linear fc2 (gate + residual)",
-    "head (layernorm + projection)", "unpatchify + guidance + mean", "drafter fusion layer", "spec_verify",
+    "head (layernorm + projection)", "guidance + mean", "drafter fusion layer",
+    "spec_verify_fused (guidance + mean + verification)",
     "round control"};
 
 struct ProfRec { int cls; double work; cudaEvent_t e0, e1; };
@@ -88,7 +89,7 @@ Workspace plan(const free_ctx* c, int n, void* base) {
     w.att = take(M * D * as);
     w.hmlp = take(M * (size_t)c->F * as);
     w.emb = take(M * D * as);
-    w.head_out = (float*)take(M * c->out_dim * 4);
+    w.head_out = (float*)take(S * (size_t)c->d_latent * 4);     // noise prediction of every stream as images
     w.fin_split = take((size_t)c->out_dim * D * 2 * 2);       // regrouped head matrix: bf16 hi and lo planes, or one fp32 copy
     w.fin_bias = (float*)take((size_t)c->out_dim * 4);
     const size_t dl = c->d_latent;
@@ -208,15 +209,17 @@ int run_blocks(const free_ctx* c, const Workspace& w, const Stack& st, int S, cu
 // the error of the noise prediction from 1.1e-2 to 1.4e-2 of the 2e-2 bound, so activations and weights are each
 // split into bf16 hi + lo planes and  y W^T ~ y_hi W_hi^T + y_lo W_hi^T + y_hi W_lo^T  (the dropped lo*lo term
 // is 2^-16 relative) is accumulated in fp32 by three small GEMMs.
-// Output: `out` [S * n_tok, c_out*p*p] with the per-token vector regrouped to (channel, row-in-patch, column-in-patch):
-// the head matrix and bias are copied with their rows in that order first.
+// Output: `out` fp32 [S, C, H, W]: the noise channels of every sequence as images.  The head matrix and bias are first
+// copied with their rows regrouped to (channel, row-in-patch, column-in-patch); the GEMM's epilogue drops the
+// remaining (variance) channels and scatters each token's vector into its patch (unpatchify fused into the store).
 int run_head(const free_ctx* c, const Workspace& w, const Stack& st, int S, float* out, cudaStream_t s) {
     const free_model_desc& m = c->m;
     const int D = m.D, T = c->n_tok, M = S * T, N = c->out_dim;
     Scope prof(c, PC_HEAD, 2.0 * M * D * N, s);
     LinearArgs a;
     a.M = M; a.N = N; a.K = D; a.bias = w.fin_bias;
-    a.epi = EPI_BIAS; a.out_dtype = FREE_FP32; a.out = out;
+    a.epi = EPI_UNPATCH; a.out_dtype = FREE_FP32; a.out = out;
+    a.n_tok = T; a.img_C = m.C; a.img_H = m.H; a.img_W = m.W; a.img_p = m.patch;
     if (m.dtype == FREE_BF16 && linear_bf16_supported(N, D)) {
         void* w_hi = w.fin_split;
         void* w_lo = (char*)w.fin_split + (size_t)N * D * 2;
@@ -227,7 +230,7 @@ int run_head(const free_ctx* c, const Workspace& w, const Stack& st, int S, floa
         a.err = w.err;
         a.A = y_hi; a.W = w_hi;
         FREE_TRY(linear_bf16(a, s));                              // bias + y_hi W_hi^T
-        a.epi = EPI_GATE_RESIDUAL; a.bias = nullptr; a.out = nullptr; a.resid = out; a.gate = nullptr; a.rows_per_seq = T;
+        a.epi = EPI_UNPATCH_ACC; a.bias = nullptr;
         a.A = y_lo; a.W = w_hi;
         FREE_TRY(linear_bf16(a, s));                              // += y_lo W_hi^T
         a.A = y_hi; a.W = w_lo;
@@ -245,7 +248,7 @@ struct PassIO {
     float* mean_out; long long mean_stride;
     float* eps_out;
     void* feat_out;
-    float* head_raw;            // if set: the pass ends with the head's output written here (no guidance, no mean)
+    float* head_raw;            // if set: the pass ends with the noise prediction of every stream [S, C, H, W] written here
     // sampling (optional): sample = mean + sigma * noise
     const float* noise; long long noise_stride;
     float* sample_out; long long sample_stride;
@@ -263,7 +266,7 @@ int tail(const free_ctx* c, const Workspace& w, int n_states, int G, float cfg, 
          const PassIO& io, cudaStream_t s) {
     const free_model_desc& m = c->m;
     Scope prof(c, PC_TAIL, (double)n_states * c->d_latent * 4 * 3, s);
-    return head_to_mean(n_states, G, m.C, m.H, m.W, m.patch, m.c_out, cfg, sch->N, w.head_out, io.x_in, io.x_stride,
+    return head_to_mean(n_states, G, c->d_latent, cfg, sch->N, w.head_out, io.x_in, io.x_stride,
                         io.t_idx, sch->coef_x, sch->coef_eps, sch->sigma2, io.mean_out, io.mean_stride,
                         io.eps_out, c->d_latent, io.noise, io.noise_stride, io.sample_out, io.sample_stride,
                         io.sample_out2, io.sample2_stride, io.sample2_mask, s);
@@ -481,16 +484,16 @@ extern "C" int dit_verify_pass(free_ctx* c, int n_states, const float* x_in, con
 }
 
 extern "C" int dit_verify_pass_raw(free_ctx* c, int n_states, const float* x_in, const int32_t* t_idx, const int32_t* labels,
-                                   int guidance, const free_schedule* sch, float* head_out, void* feat_out,
+                                   int guidance, const free_schedule* sch, float* eps_out, void* feat_out,
                                    void* ws, size_t ws_bytes, void* stream) {
-    if (!x_in || !t_idx || !labels || !head_out) return FREE_ERR_ARG;
+    if (!x_in || !t_idx || !labels || !eps_out) return FREE_ERR_ARG;
     FREE_TRY(check_common(c, n_states, sch, ws, ws_bytes));
-    if (!free_aligned16(x_in) || !free_aligned16(head_out) || !free_aligned16(feat_out)) return FREE_ERR_ALIGN;
+    if (!free_aligned16(x_in) || !free_aligned16(eps_out) || !free_aligned16(feat_out)) return FREE_ERR_ALIGN;
     const Workspace w = plan(c, n_states, ws);
     FREE_CUDA_TRY(cudaMemsetAsync(w.err, 0, 4, reinterpret_cast<cudaStream_t>(stream)));
     PassIO io{};
     io.x_in = x_in; io.x_stride = c->d_latent; io.t_idx = t_idx; io.labels = labels;
-    io.feat_out = feat_out; io.head_raw = head_out;
+    io.feat_out = feat_out; io.head_raw = eps_out;
     return target_pass(c, w, n_states, guidance ? 2.f : 0.f, sch, io, reinterpret_cast<cudaStream_t>(stream));
 }
 
@@ -566,9 +569,8 @@ int one_round(const free_ctx* c, const Workspace& w, const RoundIO& r, cudaStrea
         // (4) guidance, the means m_{a+1..a+K} and the sequential verification with the first-rejection break in one
         //     kernel; the finalised state replaces x_cur
         const int G = (r.cfg > 0.f && r.cfg != 1.f) ? 2 : 1;
-        const free_model_desc& m = c->m;
         { Scope p(c, PC_VERIFY, (double)B * ((2.0 + G) * K + 2) * d * 4, s);
-          FREE_TRY(spec_verify_fused_launch(B, K, m.C, m.H, m.W, m.patch, m.c_out, G, r.cfg, w.head_out, w.pack_in, (long long)K * d,
+          FREE_TRY(spec_verify_fused_launch(B, K, d, G, r.cfg, w.head_out, w.pack_in, (long long)K * d,
                                             w.m_draft, w.x_draft, w.cx_bk, w.ce_bk, w.sigma2_bk, w.lam_bk, w.u_bk, w.nv, 0,
                                             w.x_cur, w.n_acc, nullptr, nullptr, s)); }
     }

@@ -16,6 +16,7 @@ struct SimtArgs {
     void* out; long long ldo;
     float* resid; const float* gate; long long gate_stride; int rows_per_seq;
     const float* emb; const int32_t* emb_idx;
+    int n_tok, img_C, img_H, img_W, img_p;
 };
 
 __global__ void __launch_bounds__(256) linear_fp32_kernel(SimtArgs a) {
@@ -59,6 +60,15 @@ __global__ void __launch_bounds__(256) linear_fp32_kernel(SimtArgs a) {
                 a.resid[(long long)gm * a.N + gn] += g * v;
                 continue;
             }
+            if (a.epi == EPI_UNPATCH || a.epi == EPI_UNPATCH_ACC) {     // head: token vectors scattered into images
+                const int p = a.img_p, gw = a.img_W / p, ch = gn / (p * p), pr = (gn % (p * p)) / p, pc = gn % p;
+                if (ch >= a.img_C) continue;
+                const int seq = gm / a.n_tok, tok = gm % a.n_tok;
+                float* dst = reinterpret_cast<float*>(a.out) +
+                             (((long long)seq * a.img_C + ch) * a.img_H + (tok / gw) * p + pr) * a.img_W + (tok % gw) * p + pc;
+                *dst = (a.epi == EPI_UNPATCH_ACC ? *dst : 0.f) + v;
+                continue;
+            }
             if (a.epi == EPI_BIAS_GELU) v = free_gelu_tanh(v);
             else if (a.epi == EPI_BIAS_SILU) v = free_silu(v);
             else if (a.epi == EPI_BIAS_EMB_SILU) v = free_silu(v + a.emb[(long long)a.emb_idx[gm] * a.N + gn]);
@@ -72,12 +82,15 @@ __global__ void __launch_bounds__(256) linear_fp32_kernel(SimtArgs a) {
 
 int linear_fp32(const LinearArgs& l, cudaStream_t s) {
     if (l.M < 1 || l.N < 1 || l.K < 1 || !l.A || !l.W) return FREE_ERR_ARG;
-    if (l.epi == EPI_QKV_HEADS) return FREE_ERR_UNSUPPORTED;
+    if (l.epi == EPI_QKV_HEADS || l.epi == EPI_QKV_TOKV) return FREE_ERR_UNSUPPORTED;
+    if ((l.epi == EPI_UNPATCH || l.epi == EPI_UNPATCH_ACC) &&
+        (l.img_p < 1 || l.img_C < 1 || l.img_H % l.img_p || l.img_W % l.img_p || l.n_tok != (l.img_H / l.img_p) * (l.img_W / l.img_p) ||
+         l.M % l.n_tok || l.out_dtype != FREE_FP32)) return FREE_ERR_ARG;
     if (l.epi == EPI_GATE_RESIDUAL ? !l.resid : !l.out) return FREE_ERR_ARG;
     if (l.epi == EPI_BIAS_EMB_SILU && (!l.emb || !l.emb_idx)) return FREE_ERR_ARG;
     SimtArgs a{l.M, l.N, l.K, (const float*)l.A, l.lda ? l.lda : l.K, (const float*)l.W, l.ldw ? l.ldw : l.K, l.bias,
                l.epi, l.out_dtype, l.out, l.ldo ? l.ldo : l.N, l.resid, l.gate, l.gate_stride,
-               l.rows_per_seq > 0 ? l.rows_per_seq : 1, l.emb, l.emb_idx};
+               l.rows_per_seq > 0 ? l.rows_per_seq : 1, l.emb, l.emb_idx, l.n_tok, l.img_C, l.img_H, l.img_W, l.img_p};
     dim3 grid((l.N + TN - 1) / TN, (l.M + TM - 1) / TM);
     linear_fp32_kernel<<<grid, 256, 0, s>>>(a);
     return free_check_launch();

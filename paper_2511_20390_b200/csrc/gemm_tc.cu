@@ -34,6 +34,7 @@ struct TcArgs {
     const float* emb; const int32_t* emb_idx;
     int heads, d_head, d_pad, n_tok;
     __nv_bfloat16 *q, *k, *vt;
+    int img_C, img_H, img_W, img_p;
     uint32_t* err;
 };
 
@@ -124,6 +125,35 @@ __device__ __forceinline__ void epilogue_chunk(const TcArgs& a, int row, int n0,
                 for (int i = 0; i < 8; ++i) dst[(long long)i * T] = __float2bfloat16(v[8 * g + i]);
                 if (c + 8 == dh)
                     for (int z = dh; z < dp; ++z) a.vt[(sh * dp + z) * T + tok] = __float2bfloat16(0.f);
+            }
+        }
+        return;
+    }
+    if (EPI == EPI_UNPATCH || EPI == EPI_UNPATCH_ACC) {
+        // the thread's token: its patch is p rows of p pixels per channel; consecutive threads hold consecutive tokens of a
+        // patch row, so that the stores of a warp to one image row are contiguous
+        const int p = a.img_p, gw = a.img_W / p, pp = p * p;
+        const int seq = row / a.n_tok, tok = row % a.n_tok, trow = tok / gw, tcol = tok % gw;
+        float* img = reinterpret_cast<float*>(a.out) + (long long)seq * a.img_C * a.img_H * a.img_W;
+        if (p == 2) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+                const int n = n0 + i, ch = n >> 2, pr = (n >> 1) & 1;
+                if (ch < a.img_C) {
+                    float2* dst = reinterpret_cast<float2*>(img + ((long long)ch * a.img_H + trow * 2 + pr) * a.img_W + tcol * 2);
+                    float2 o = make_float2(v[i], v[i + 1]);
+                    if (EPI == EPI_UNPATCH_ACC) { const float2 old = *dst; o.x += old.x; o.y += old.y; }
+                    *dst = o;
+                }
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const int n = n0 + i, ch = n / pp, pr = (n % pp) / p, pc = n % p;
+                if (ch < a.img_C) {
+                    float* dst = img + ((long long)ch * a.img_H + trow * p + pr) * a.img_W + tcol * p + pc;
+                    *dst = (EPI == EPI_UNPATCH_ACC ? *dst : 0.f) + v[i];
+                }
             }
         }
         return;
@@ -315,6 +345,10 @@ static int validate_epilogue(const LinearArgs& l, long long ldo) {
         case EPI_QKV_TOKV:
             return (!l.out || !l.vt || !free_aligned16(l.out) || ldo % 8 || l.heads < 1 || l.d_head % 8 || l.d_pad % 8 || l.d_pad < l.d_head ||
                     l.n_tok < 1 || l.N != 3 * l.heads * l.d_head || l.M % l.n_tok) ? FREE_ERR_ARG : FREE_OK;
+        case EPI_UNPATCH: case EPI_UNPATCH_ACC:
+            return (!l.out || !free_aligned16(l.out) || l.out_dtype != FREE_FP32 || l.img_p < 1 || l.img_C < 1 || l.img_H % l.img_p ||
+                    l.img_W % l.img_p || l.n_tok != (l.img_H / l.img_p) * (l.img_W / l.img_p) || l.M % l.n_tok ||
+                    l.N < l.img_C * l.img_p * l.img_p) ? FREE_ERR_ARG : FREE_OK;
         default:
             return FREE_ERR_ARG;
     }
@@ -343,6 +377,7 @@ int linear_bf16(const LinearArgs& l, cudaStream_t s) {
     a.emb = l.emb; a.emb_idx = l.emb_idx;
     a.heads = l.heads; a.d_head = l.d_head; a.d_pad = l.d_pad; a.n_tok = l.n_tok;
     a.q = (__nv_bfloat16*)l.q; a.k = (__nv_bfloat16*)l.k; a.vt = (__nv_bfloat16*)l.vt;
+    a.img_C = l.img_C; a.img_H = l.img_H; a.img_W = l.img_W; a.img_p = l.img_p;
     a.err = l.err;
     const size_t smem = 1024 + kCtrlBytes + (size_t)a.stages * stage_bytes;
 
@@ -364,6 +399,10 @@ int linear_bf16(const LinearArgs& l, cudaStream_t s) {
             return launch<EPI_GATE_RESIDUAL, false>(mA, mW, a, smem, s);
         case EPI_QKV_HEADS:
             return launch<EPI_QKV_HEADS, true>(mA, mW, a, smem, s);
+        case EPI_UNPATCH:
+            return launch<EPI_UNPATCH, false>(mA, mW, a, smem, s);
+        case EPI_UNPATCH_ACC:
+            return launch<EPI_UNPATCH_ACC, false>(mA, mW, a, smem, s);
         default:
             return FREE_ERR_ARG;
     }

@@ -12,6 +12,8 @@ enum {
     EPI_BIAS_EMB_SILU = 4,                        // out = silu(acc + bias + emb[emb_idx[row], n])
     EPI_QKV_HEADS = 5,                            // bf16 only: scatter (acc + bias) into head-major q, k and v^T
     EPI_QKV_TOKV = 6,                             // bf16 only (CTA-pair kernel): q and k token-major into out[M, 2D], v^T head-major
+    EPI_UNPATCH = 7,                              // head: (acc + bias) of the first img_C channels scattered into images (see LinearArgs)
+    EPI_UNPATCH_ACC = 8,                          // the same, added to what the images hold
 };
 
 struct LinearArgs {
@@ -28,6 +30,9 @@ struct LinearArgs {
     // EPI_QKV_HEADS
     int heads = 0, d_head = 0, d_pad = 0, n_tok = 0;
     void* q = nullptr; void* k = nullptr; void* vt = nullptr;
+    // EPI_UNPATCH[_ACC]: row = seq * n_tok + token (tokens row-major over the patch grid), column = (ch * p + pr) * p + pc;
+    // out is fp32 [n_seq, img_C, img_H, img_W], element (seq, ch, trow * p + pr, tcol * p + pc); columns with ch >= img_C are dropped
+    int img_C = 0, img_H = 0, img_W = 0, img_p = 0;
     uint32_t* err = nullptr;                      // device error word (tensor-core path)
 };
 
@@ -68,17 +73,18 @@ int ln_modulate_split(int M, int D, int rows_per_seq, const float* x, const floa
 // head matrix [p*p*c_out, D] and bias with rows regrouped to (channel, row-in-patch, column-in-patch); split: bf16 hi / lo
 // planes into out0 / lo, else an fp32 copy into out0
 int head_weights(bool split, int p, int c_out, int D, const float* w, const float* b, void* out0, void* lo, float* b_out, cudaStream_t s);
-int head_to_mean(int n_states, int G, int C, int H, int W, int p, int c_out, float cfg_scale, int N_sched,
-                 const float* head_out /*[S*n_tok, c_out*p*p], vector order (channel, row, col)*/, const float* x_in, long long x_stride,
+// head_out [n_states, G, d]: the noise prediction of every stream as images (written by the head's EPI_UNPATCH epilogue)
+int head_to_mean(int n_states, int G, int d, float cfg_scale, int N_sched,
+                 const float* head_out, const float* x_in, long long x_stride,
                  const int32_t* t_idx, const float* coef_x, const float* coef_eps, const float* sigma2,
                  float* mean_out, long long mean_stride, float* eps_out, long long eps_stride,
                  const float* noise, long long noise_stride, float* sample_out, long long sample_stride,
                  float* sample_out2, long long sample2_stride, const int32_t* sample2_mask, cudaStream_t s);
 
-// ---- verification from the head's output (verify_fused.cu) -------------------------------------
+// ---- verification from the noise predictions (verify_fused.cu) ----------------------------------
 // As the public spec_verify_fused, with a row stride (elements) for x_first.
-int spec_verify_fused_launch(int B, int K, int C, int H, int W, int patch, int c_out, int G, float cfg_scale,
-                             const float* head_out, const float* x_first, long long x_first_stride,
+int spec_verify_fused_launch(int B, int K, long long d, int G, float cfg_scale,
+                             const float* eps, const float* x_first, long long x_first_stride,
                              const float* m_draft, const float* x_draft, const float* coef_x, const float* coef_eps,
                              const float* sigma2, const float* lambda, const float* u, const int32_t* n_valid, int chunk,
                              float* x_out, int32_t* n_accept, float* logratio_out, float* means_out, cudaStream_t s);

@@ -247,7 +247,7 @@ __global__ void convert_kernel(long long n, const float* __restrict__ x, T* __re
 // eps = eps_u + w (eps_c - eps_u).  mean = coef_x[t] x - coef_eps[t] eps.  Optionally draws the next
 // state sample = mean + sqrt(sigma2[t]) noise (drafter step / target step of the sampling loop).
 struct TailArgs {
-    int n_states, G, C, H, W, p, c_out, N_sched;
+    int n_states, G, d, N_sched;
     float cfg_scale;
     const float* head_out; const float* x_in; long long x_stride;
     const int32_t* t_idx; const float *coef_x, *coef_eps, *sigma2;
@@ -258,18 +258,16 @@ struct TailArgs {
     float* sample_out2; long long sample2_stride; const int32_t* sample2_mask;
 };
 
+// Guidance, the reverse-transition mean (Eq. ddpm_update) and optionally the sample, elementwise over the images the
+// head wrote: head_out [n_states, G, d].
 __global__ void __launch_bounds__(256) head_to_mean_kernel(TailArgs a) {
-    const int d = a.C * a.H * a.W;
-    const int gw = a.W / a.p, n_tok = (a.H / a.p) * gw, od = a.p * a.p * a.c_out;
+    const int d = a.d;
     const long long total = (long long)a.n_states * d;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
         const int st = (int)(i / d), e = (int)(i % d);
-        const int c = e / (a.H * a.W), yy = (e / a.W) % a.H, xx = e % a.W;
-        const int tok = (yy / a.p) * gw + xx / a.p;
-        const int vec = (c * a.p + yy % a.p) * a.p + xx % a.p;
-        float eps = a.head_out[((long long)(st * a.G) * n_tok + tok) * od + vec];
+        float eps = a.head_out[(long long)st * a.G * d + e];
         if (a.G == 2) {
-            const float eu = a.head_out[((long long)(st * a.G + 1) * n_tok + tok) * od + vec];
+            const float eu = a.head_out[((long long)st * a.G + 1) * d + e];
             eps = eu + a.cfg_scale * (eps - eu);
         }
         int t = a.t_idx[st];
@@ -383,16 +381,16 @@ int convert_rows(int out_dtype, long long n, const float* x, void* y, cudaStream
     return free_check_launch();
 }
 
-int head_to_mean(int n_states, int G, int C, int H, int W, int p, int c_out, float cfg_scale, int N_sched,
+int head_to_mean(int n_states, int G, int d, float cfg_scale, int N_sched,
                  const float* head_out, const float* x_in, long long x_stride,
                  const int32_t* t_idx, const float* coef_x, const float* coef_eps, const float* sigma2,
                  float* mean_out, long long mean_stride, float* eps_out, long long eps_stride,
                  const float* noise, long long noise_stride, float* sample_out, long long sample_stride,
                  float* sample_out2, long long sample2_stride, const int32_t* sample2_mask, cudaStream_t s) {
-    TailArgs a{n_states, G, C, H, W, p, c_out, N_sched, cfg_scale, head_out, x_in, x_stride, t_idx, coef_x, coef_eps, sigma2,
+    TailArgs a{n_states, G, d, N_sched, cfg_scale, head_out, x_in, x_stride, t_idx, coef_x, coef_eps, sigma2,
                mean_out, mean_stride, eps_out, eps_stride, noise, noise_stride, sample_out, sample_stride,
                sample_out2, sample2_stride, sample2_mask};
-    const long long total = (long long)n_states * C * H * W;
+    const long long total = (long long)n_states * d;
     const unsigned grid = (unsigned)((total + 255) / 256 > 148 * 8 ? 148 * 8 : (total + 255) / 256);
     head_to_mean_kernel<<<grid, 256, 0, s>>>(a);
     return free_check_launch();

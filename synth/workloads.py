@@ -57,18 +57,17 @@ def pack_states(seed: int, B: int, K: int, d_shape, n_sched: int, n_classes: int
     return x, t_idx, labels
 
 
-def head_verifier_inputs(seed: int, B: int, K: int, G: int, n_tok: int, vec: int, d_shape, s: float,
-                         sigma2: np.ndarray, head_std: float = 1.0):
-    """Operands of a verification that starts from a network's raw per-token output.
+def eps_verifier_inputs(seed: int, B: int, K: int, G: int, d_shape, s: float, sigma2: np.ndarray, eps_std: float = 1.0):
+    """Operands of a verification that starts from a network's noise predictions.
 
-    head [B,K,G,n_tok,vec] is N(0, head_std^2).  The state chain is x_first ~ N(0,1) followed by the
+    eps [B,K,G,*d_shape] is N(0, eps_std^2).  The state chain is x_first ~ N(0,1) followed by the
     drafts themselves: each draft mean is its predecessor in the chain plus N(0, s^2) noise, each
     draft sample its draft mean plus sqrt(sigma2[b,k]) * N(0,1); uniforms are in (0,1).
-    Returns fp32 arrays head, x_first [B,*d_shape], m_hat, x_hat [B,K,*d_shape] and u [B,K].
+    Returns fp32 arrays eps, x_first [B,*d_shape], m_hat, x_hat [B,K,*d_shape] and u [B,K].
     """
     sigma2 = np.broadcast_to(np.asarray(sigma2, dtype=np.float64), (B, K))
     d_shape = tuple(d_shape)
-    head = normal(seed, 41, (B, K, G, n_tok, vec), std=head_std)
+    eps = normal(seed, 41, (B, K, G) + d_shape, std=eps_std)
     x_first = normal(seed, 42, (B,) + d_shape)
     n = normal(seed, 43, (B, K) + d_shape)
     z = normal(seed, 44, (B, K) + d_shape)
@@ -80,4 +79,4 @@ def head_verifier_inputs(seed: int, B: int, K: int, G: int, n_tok: int, vec: int
         x_hat[:, k] = m_hat[:, k] + np.sqrt(sigma2[:, k]).astype(np.float32).reshape((B,) + (1,) * len(d_shape)) * z[:, k]
         prev = x_hat[:, k]
     u = uniform01(seed, 45, (B, K))
-    return head, x_first, m_hat, x_hat, u
+    return eps, x_first, m_hat, x_hat, u

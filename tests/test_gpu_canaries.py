@@ -88,3 +88,25 @@ def test_verifier_stays_in_bounds():
     free.spec_verify(cu(m), cu(mh), cu(xh), cu(s2), cu(u), x_out=x_out.t.view(B, d), n_accept=n_acc.t[:B])
     torch.cuda.synchronize()
     assert x_out.intact() and n_acc.intact()
+
+
+def test_fused_verifier_stays_in_bounds():
+    import paper_2511_20390_b200 as free
+    B, K, G, shape = 5, 3, 2, (4, 32, 33)                  # d = 4224: ragged against the cluster stride
+    d = int(np.prod(shape))
+    eps, x_first, mh, xh, u = synth.eps_verifier_inputs(4, B, K, G, shape, 0.01, np.full((B, K), 0.02), eps_std=0.1)
+    cu = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(torch.float32).cuda()
+    one = torch.ones(B, K, device="cuda", dtype=torch.float32)
+    x_out, means, n_acc = Guarded(B * d * 4, torch.float32), Guarded(B * K * d * 4, torch.float32), Guarded(B * 4, torch.int32)
+    ell = Guarded(B * K * 4, torch.float32)
+    L = free.lib()
+    st = torch.cuda.current_stream().cuda_stream
+    ts = [cu(eps), cu(x_first), cu(mh), cu(xh)]
+    ce, s2, uu = 0.05 * one, 0.02 * one, cu(u)
+    for chunk in (0, 2):
+        rc = L.spec_verify_fused(B, K, d, G, 4.0, ts[0].data_ptr(), ts[1].data_ptr(), ts[2].data_ptr(), ts[3].data_ptr(),
+                                 one.data_ptr(), ce.data_ptr(), s2.data_ptr(), None, uu.data_ptr(), None, chunk,
+                                 x_out.t.data_ptr(), n_acc.t.data_ptr(), ell.t.data_ptr(), means.t.data_ptr(), st)
+        assert rc == 0
+        torch.cuda.synchronize()
+        assert x_out.intact() and means.intact() and n_acc.intact() and ell.intact()

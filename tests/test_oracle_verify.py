@@ -177,79 +177,67 @@ def test_sigma_must_be_positive():
         V.verification(np.zeros(2), np.ones(2), 0.0, np.zeros(2), 0.5)
 
 
-# ----------------------------------------------------------------------------- verification from the raw head output
-def _scatter_head(eps_img, p):
-    """Brute force: place eps_img[g, c, h, w] into the per-token vectors one element at a time."""
-    G, c_out, H, W = eps_img.shape
-    gw = W // p
-    tok = np.zeros((G, (H // p) * gw, c_out * p * p))
-    for g in range(G):
-        for c in range(c_out):
-            for h in range(H):
-                for w in range(W):
-                    tok[g, (h // p) * gw + w // p, (c * p + h % p) * p + w % p] = eps_img[g, c, h, w]
-    return tok
-
-
-@pytest.mark.parametrize("G,p,C,H,W", [(2, 2, 4, 4, 6), (1, 2, 3, 6, 4), (2, 1, 2, 3, 5), (2, 3, 1, 6, 9)])
-def test_means_from_head_output_against_elementwise_loops(G, p, C, H, W):
-    rng = np.random.default_rng(G * 100 + p * 10 + C)
-    K, c_out, w_cfg = 3, 2 * C, 2.5
-    eps_img = rng.standard_normal((K, G, c_out, H, W))
-    head = np.stack([_scatter_head(eps_img[k], p) for k in range(K)])
-    x_first = rng.standard_normal((C, H, W))
-    x_hat = rng.standard_normal((K, C, H, W))
+# ----------------------------------------------------------------------------- verification from the noise predictions
+@pytest.mark.parametrize("G,shape", [(2, (4, 4, 6)), (1, (3, 5)), (2, (7,))])
+def test_means_from_stream_eps_against_elementwise_loops(G, shape):
+    rng = np.random.default_rng(G * 100 + len(shape))
+    K, w_cfg = 3, 2.5
+    eps = rng.standard_normal((K, G) + shape)
+    x_first = rng.standard_normal(shape)
+    x_hat = rng.standard_normal((K,) + shape)
     cx, ce = rng.uniform(1.0, 1.1, K), rng.uniform(0.01, 0.2, K)
-    got = V.means_from_head_output(head, x_first, x_hat, cx, ce, w_cfg, C, H, W, p)
+    got = V.means_from_stream_eps(eps, x_first, x_hat, cx, ce, w_cfg)
     for k in range(K):
         x_k = x_first if k == 0 else x_hat[k - 1]
-        for c in range(C):
-            for h in range(H):
-                for w in range(W):
-                    e = eps_img[k, 0, c, h, w]
-                    if G == 2:
-                        e = eps_img[k, 1, c, h, w] + w_cfg * (eps_img[k, 0, c, h, w] - eps_img[k, 1, c, h, w])
-                    assert abs(got[k, c, h, w] - (cx[k] * x_k[c, h, w] - ce[k] * e)) < 1e-13
+        for idx in np.ndindex(*shape):
+            e = eps[(k, 0) + idx]
+            if G == 2:
+                e = eps[(k, 1) + idx] + w_cfg * (eps[(k, 0) + idx] - eps[(k, 1) + idx])
+            assert abs(got[(k,) + idx] - (cx[k] * x_k[idx] - ce[k] * e)) < 1e-13
 
 
-def test_means_from_head_output_special_cases():
+def test_means_from_stream_eps_special_cases():
     rng = np.random.default_rng(77)
-    K, G, C, H, W, p = 2, 2, 2, 4, 4, 2
-    head = rng.standard_normal((K, G, 4, 2 * C * p * p))
-    x_first, x_hat = rng.standard_normal((C, H, W)), rng.standard_normal((K, C, H, W))
+    K, G, shape = 2, 2, (2, 4, 4)
+    eps = rng.standard_normal((K, G) + shape)
+    x_first, x_hat = rng.standard_normal(shape), rng.standard_normal((K,) + shape)
     one, zero = np.ones(K), np.zeros(K)
     # coef_eps = 0: the mean is the packed state itself -- x_first, then the drafts shifted by one slot
-    m = V.means_from_head_output(head, x_first, x_hat, one, zero, 3.0, C, H, W, p)
+    m = V.means_from_stream_eps(eps, x_first, x_hat, one, zero, 3.0)
     assert np.array_equal(m[0], x_first) and np.array_equal(m[1], x_hat[0])
     # guidance scale 1 with two streams: the conditional stream alone; scale 0: the unconditional one
-    m1 = V.means_from_head_output(head, x_first, x_hat, zero, -one, 1.0, C, H, W, p)
-    mc = V.means_from_head_output(head[:, :1], x_first, x_hat, zero, -one, 1.0, C, H, W, p)
-    mu = V.means_from_head_output(head[:, 1:], x_first, x_hat, zero, -one, 1.0, C, H, W, p)
-    m0 = V.means_from_head_output(head, x_first, x_hat, zero, -one, 0.0, C, H, W, p)
-    assert np.allclose(m1, mc, atol=1e-15) and np.allclose(m0, mu, atol=1e-15)
-    # the variance channels (c >= C) never matter
-    head2 = head.copy().reshape(K, G, 4, 2 * C, p * p)
-    head2[:, :, :, C:] += 5.0
-    assert np.array_equal(V.means_from_head_output(head2.reshape(head.shape), x_first, x_hat, one, one, 3.0, C, H, W, p),
-                          V.means_from_head_output(head, x_first, x_hat, one, one, 3.0, C, H, W, p))
+    m1 = V.means_from_stream_eps(eps, x_first, x_hat, zero, -one, 1.0)
+    m0 = V.means_from_stream_eps(eps, x_first, x_hat, zero, -one, 0.0)
+    assert np.allclose(m1, eps[:, 0], atol=1e-15) and np.allclose(m0, eps[:, 1], atol=1e-15)
+    # one stream: the scale does not enter
+    assert np.array_equal(V.means_from_stream_eps(eps[:, :1], x_first, x_hat, one, one, 3.0),
+                          V.means_from_stream_eps(eps[:, :1], x_first, x_hat, one, one, 0.0))
+    # equal to the schedule's own mean with guided eps (two independent routes to Eq. ddpm_update)
+    from oracle import schedule as S
+    sc = S.make("respaced", 50)
+    idx = np.array([30, 29])
+    m = V.means_from_stream_eps(eps, x_first, x_hat, sc.coef_x[idx], sc.coef_eps[idx], 4.0)
+    for k in range(K):
+        guided = eps[k, 1] + 4.0 * (eps[k, 0] - eps[k, 1])
+        assert np.allclose(m[k], sc.mean(x_first if k == 0 else x_hat[k - 1], guided, int(idx[k])), atol=1e-14)
 
 
-def test_spec_verify_from_head_is_verification_of_those_means():
+def test_spec_verify_from_eps_is_verification_of_those_means():
     rng = np.random.default_rng(5)
-    B, K, G, C, H, W, p = 3, 4, 2, 2, 4, 4, 2
-    head = 0.1 * rng.standard_normal((B, K, G, 4, 2 * C * p * p))
-    x_first = rng.standard_normal((B, C, H, W))
+    B, K, G, shape = 3, 4, 2, (2, 4, 4)
+    eps = 0.1 * rng.standard_normal((B, K, G) + shape)
+    x_first = rng.standard_normal((B,) + shape)
     cx, ce = np.full((B, K), 1.01), np.full((B, K), 0.05)
     sigma2, u = np.full((B, K), 0.02), rng.uniform(0.0, 1.0, (B, K))
     # drafts built around the true means so that some are accepted and some are not
-    x_hat = np.zeros((B, K, C, H, W)); m_hat = np.zeros_like(x_hat)
+    x_hat = np.zeros((B, K) + shape); m_hat = np.zeros_like(x_hat)
     for b in range(B):
         for k in range(K):
             xk = x_first[b] if k == 0 else x_hat[b, k - 1]
-            mk = V.means_from_head_output(head[b, k:k + 1], xk, x_hat[b, :1], cx[b, k:k + 1], ce[b, k:k + 1], 2.0, C, H, W, p)[0]
+            mk = V.means_from_stream_eps(eps[b, k:k + 1], xk, x_hat[b, :1], cx[b, k:k + 1], ce[b, k:k + 1], 2.0)[0]
             m_hat[b, k] = mk + 0.03 * rng.standard_normal(mk.shape)
             x_hat[b, k] = m_hat[b, k] + np.sqrt(sigma2[b, k]) * rng.standard_normal(mk.shape)
-    x_out, n_acc, ell, means = V.spec_verify_from_head(head, x_first, m_hat, x_hat, cx, ce, 2.0, (C, H, W, p), sigma2, u)
+    x_out, n_acc, ell, means = V.spec_verify_from_eps(eps, x_first, m_hat, x_hat, cx, ce, 2.0, sigma2, u)
     assert 0 < n_acc.sum() < B * K            # a mix of outcomes
     for b in range(B):
         state = None
