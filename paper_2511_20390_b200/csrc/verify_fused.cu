@@ -66,7 +66,7 @@ __device__ __forceinline__ void accumulate4(const Row& r, long long i, double& s
 }
 
 template <int CLUSTER, bool VEC4, bool G2>
-__global__ void __launch_bounds__(kThreads, 3) spec_verify_fused_kernel(FusedArgs a) {
+__global__ void __launch_bounds__(kThreads, 4) spec_verify_fused_kernel(FusedArgs a) {
     __shared__ double warp_part[FREE_MAX_K][kWarps][2];
     __shared__ double cta_part[FREE_MAX_K][2];
     __shared__ double tot[FREE_MAX_K][2];
@@ -266,7 +266,7 @@ int spec_verify_fused_launch(int B, int K, long long d, int G, float cfg_scale,
     if (!vec) return d >= 4096 ? launch_g<4, false>(a, s) : launch_g<1, false>(a, s);
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { (void)cudaGetLastError(); sms = 148; }
-    const long long resident = 3LL * sms;                 // 256-thread CTAs of this kernel that fit on the GPU at once
+    const long long resident = 4LL * sms;                 // 256-thread CTAs of this kernel that fit on the GPU at once
     int width = d >= 8192 ? 8 : (d >= 4096 ? 4 : (d >= 2048 ? 2 : 1));
     while (width > 2 && (long long)B * width > resident) width >>= 1;
     switch (width) {
