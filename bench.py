@@ -217,10 +217,15 @@ class FusedVerifierWorkload:
         rows = np.minimum(self.K, (np.minimum(n, self.K - 1) // self.chunk + 1) * self.chunk)
         return int((rows * (self.G + 2) * self.d * 4 + 2 * self.d * 4 + 20 * rows).sum())
 
+    # DRAM bytes (read + write) of one launch at B = 64, chunk 0, from the ncu capture summarised in
+    # profiles/spec_verify_fused_kernel_K16_B64.txt; traffic is proportional to the batch
+    NCU_DRAM_BYTES_B64 = 298.2e6
+
     def roofline(self, ms_per_step, peaks):
         ach = self.bytes_examined() / 1e9 / (ms_per_step / 1e3)
+        traffic = self.NCU_DRAM_BYTES_B64 * self.B / 64.0 if self.chunk == 0 else None
         return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": ach / peaks["hbm_gbs"], "traffic": None, "kernel": "spec_verify_fused_kernel",
+                "frac": ach / peaks["hbm_gbs"], "traffic": traffic, "kernel": "spec_verify_fused_kernel",
                 "peak_source": peaks["source"]}
 
     def extra(self, ms_step, peaks):

@@ -11,7 +11,7 @@ static const char* const kProfNames[PC_N] = {
     "conditioning + modulation tables", "patch embed / feature copy", "layernorm + modulate", "linear qkv",
     "attention", "linear proj (gate + residual)", "linear fc1 + gelu", "linear fc2 (gate + residual)",
     "head (layernorm + projection)", "guidance + mean", "drafter fusion layer",
-    "spec_verify_fused (guidance + mean + verification)",
+    "spec_verify_fused (guidance, mean, verify)",
     "round control"};
 
 struct ProfRec { int cls; double work; cudaEvent_t e0, e1; };
