@@ -189,6 +189,9 @@ int spec_verify(int B, int K, int64_t d,
  *              x_out and n_accept are unchanged by this, logratio_out is NaN for drafts that were not examined, and
  *              FREE_ERR_SIGMA is reported only for examined drafts.
  *   x_out, n_accept, logratio_out   as for spec_verify (x_out may not alias x_first or x_draft)
+ *   dist2_out  DEVICE fp32 [B, K] or NULL: |m_hat - m|^2 of every examined draft (NaN for the others).  Both means come
+ *              from the same packed state, so |eps_pred - eps_ref| = sqrt(dist2) / coef_eps: the prediction deviation
+ *              that Sec. 3.4 tracks.
  *   means_out  DEVICE fp32 [B, K, d] or NULL: the target means of the examined drafts, rounded to fp32 (diagnostic)
  * No workspace.  Errors: ARG (null pointer, G not 1 or 2), SHAPE, ALIGN, CUDA.
  */
@@ -196,7 +199,7 @@ int spec_verify_fused(int B, int K, int64_t d, int G, float cfg_scale,
                       const float* eps, const float* x_first, const float* m_draft, const float* x_draft,
                       const float* coef_x, const float* coef_eps, const float* sigma2, const float* lambda,
                       const float* u, const int32_t* n_valid, int chunk,
-                      float* x_out, int32_t* n_accept, float* logratio_out, float* means_out, void* stream);
+                      float* x_out, int32_t* n_accept, float* logratio_out, float* dist2_out, float* means_out, void* stream);
 
 /*
  * draft_step -- one step of feature-level autoregression (Sec. 3.1; Alg. 1, drafting loop) for
@@ -251,6 +254,35 @@ int sample_trajectory(free_ctx* ctx, int B,
                            const float* noise_target, const float* noise_draft, const float* uniforms,
                            float* x_final, free_traj_stats* stats,
                            void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * free_uncertainty_profile -- the offline run of Sec. 3.4: Algorithm 1 (as sample_trajectory, strict or with the given
+ * lambda) with the context's drafter proposing and the target verifying, recording for every EXAMINED draft (the
+ * accepted ones and the rejected one of each round) the prediction deviation |eps_pred - eps_ref|_2 and the acceptance
+ * probability min(1, e^ell), averaged per transition.  Both noise predictions refer to the same packed state, so the
+ * deviation is |m_hat - m| / coef_eps, taken from the verifier's own sums.  (The paper runs the DiT against itself; a
+ * DiT has no feature input, so here the proposer is whatever drafter the context holds.)
+ *   eps_delta, accept_prob   HOST double [N], index n-1 for transition n; 0 where count is 0
+ *   count                    HOST int64 [N]: examined drafts per transition (transition 1 and the last are never drafted)
+ *   params->K >= 1; other arguments as for sample_trajectory.  Blocks until done.
+ */
+int free_uncertainty_profile(free_ctx* ctx, int B, const float* x0, const int32_t* labels,
+                             const free_schedule* sched, const free_spec_params* params,
+                             const float* noise_target, const float* noise_draft, const float* uniforms,
+                             double* eps_delta, double* accept_prob, int64_t* count,
+                             void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * free_fit_lambda_profile -- relaxation table lambda_n from measured deviations (Sec. 3.4: a smooth, monotonically
+ * increasing curve fitted to eps_delta, inverted and rescaled to [0, 1]).  Host-only.  Steps: transitions without a
+ * measurement (count == 0, NaN or negative) take the nearest measured value; weighted least-squares non-decreasing fit
+ * (pool adjacent violators, weights = count, or 1 when count is NULL); centred moving average over 2*window+1 points
+ * with the ends held (keeps the curve non-decreasing); lambda_n = g_1 / g_n, which is 1 at the first transition,
+ * non-increasing, in (0, 1], and makes lambda_n * g_n constant (a uniform scaled discrepancy).  g_n = 0 gives 1.
+ *   eps_delta HOST double [N]; count HOST int64 [N] or NULL; lambda_out HOST fp32 [N] (the table of free_spec_params)
+ * Errors: ARG, SHAPE (N < 1, window < 0, nothing measured).
+ */
+int free_fit_lambda_profile(const double* eps_delta, const int64_t* count, int N, int window, float* lambda_out);
 
 /*
  * spec_round -- the body of Algorithm 1's loop, once: for every sample b whose cursor[b] <= N (cursor = index of

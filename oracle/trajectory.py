@@ -19,13 +19,15 @@ from . import verify
 
 
 def sample(x0, N, K, target_fn, draft_fn, sigma2, noise_target, noise_draft, uniforms,
-           lam=None, trace=None):
+           lam=None, trace=None, observe=None):
     """Run one trajectory.
 
     target_fn(x, s)              -> (mean, feature)          one target evaluation at schedule index s
     target_fn.packed(xs, ss)     -> means                     optional batched form (else called per state)
     draft_fn(x_prev, f_prev, s)  -> (mean_hat, feature_next)
     sigma2[s]; noise_target[n-1], noise_draft[n-1] of x0's shape; uniforms[n-1]; lam[n-1] or None.
+    observe(t, m_hat_t, m_t, ell), if given, is called for every examined draft (used by the offline
+    uncertainty run of Sec. 3.4).
     K == 0 is the plain sequential sampler.  Returns (x_N, stats).
     """
     x = np.asarray(x0, np.float64)
@@ -60,6 +62,8 @@ def sample(x0, N, K, target_fn, draft_fn, sigma2, noise_target, noise_draft, uni
             x, ok, ell = verify.verification(m_hat[t], m[t], sigma2[N - t], x_hat[t], uniforms[t - 1], lam_t)
             if trace is not None:
                 trace.append((t, ok, ell))
+            if observe is not None:
+                observe(t, m_hat[t], m[t], ell)
             j = t
             if not ok:
                 stats["rejected"] += 1

@@ -72,7 +72,7 @@ _SIGNATURES = {
     "dit_verify_pass_raw": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                                       C.POINTER(ScheduleDesc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "spec_verify": (C.c_int, [C.c_int, C.c_int, C.c_int64] + [C.c_void_p] * 11),
-    "spec_verify_fused": (C.c_int, [C.c_int, C.c_int, C.c_int64, C.c_int, C.c_float] + [C.c_void_p] * 10 + [C.c_int] + [C.c_void_p] * 5),
+    "spec_verify_fused": (C.c_int, [C.c_int, C.c_int, C.c_int64, C.c_int, C.c_float] + [C.c_void_p] * 10 + [C.c_int] + [C.c_void_p] * 6),
     "draft_step": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
                              C.POINTER(ScheduleDesc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                              C.c_void_p, C.c_size_t, C.c_void_p]),
@@ -82,6 +82,10 @@ _SIGNATURES = {
     "free_spec_round": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(ScheduleDesc),
                                   C.POINTER(SpecParams), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                   C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "free_uncertainty_profile": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.POINTER(ScheduleDesc),
+                                           C.POINTER(SpecParams), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "free_fit_lambda_profile": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p]),
     "free_profile_begin": (C.c_int, [C.c_void_p]),
     "free_profile_end": (C.c_int, [C.c_void_p, C.POINTER(ProfEntry), C.c_int, C.POINTER(C.c_int)]),
     "free_op_linear_workspace_bytes": (C.c_size_t, []),
@@ -154,10 +158,10 @@ def spec_verify(m, m_hat, x_hat, sigma2, u, lam=None, n_valid=None, want_lograti
 
 
 def spec_verify_fused(eps, x_first, m_hat, x_hat, coef_x, coef_eps, sigma2, u, cfg_scale, lam=None,
-                      n_valid=None, chunk=0, want_logratio=False, want_means=False, x_out=None, n_accept=None):
+                      n_valid=None, chunk=0, want_logratio=False, want_means=False, want_dist2=False, x_out=None, n_accept=None):
     """Verification straight from the packed pass's noise predictions (guidance, Eq. ddpm_update and Algorithm 2 in
     one kernel).  eps: CUDA fp32 [B,K,G,d...]; x_first [B,d...]; m_hat, x_hat [B,K,d...]; coef_x, coef_eps, sigma2, u,
-    lam: [B,K]; chunk > 0 enables the early exit.  Returns (x_out, n_accept[, ell][, means])."""
+    lam: [B,K]; chunk > 0 enables the early exit.  Returns (x_out, n_accept[, ell][, means][, dist2])."""
     B, K, G = eps.shape[:3]
     d = int(np.prod(eps.shape[3:]))
     for t in (eps, x_first, m_hat, x_hat, coef_x, coef_eps, sigma2, u):
@@ -169,13 +173,27 @@ def spec_verify_fused(eps, x_first, m_hat, x_hat, coef_x, coef_eps, sigma2, u, c
         n_accept = torch.empty(B, dtype=torch.int32, device=dev)
     ell = torch.empty((B, K), dtype=torch.float32, device=dev) if want_logratio else None
     means = torch.zeros((B, K) + tuple(eps.shape[3:]), dtype=torch.float32, device=dev) if want_means else None
+    dist2 = torch.empty((B, K), dtype=torch.float32, device=dev) if want_dist2 else None
     code = lib().spec_verify_fused(B, K, d, G, float(cfg_scale), _ptr(eps), _ptr(x_first),
                                    _ptr(m_hat), _ptr(x_hat), _ptr(coef_x), _ptr(coef_eps), _ptr(sigma2),
                                    _ptr(None if lam is None else _dev(lam, torch.float32)), _ptr(u),
                                    _ptr(None if n_valid is None else _dev(n_valid, torch.int32)), int(chunk),
-                                   _ptr(x_out), _ptr(n_accept), _ptr(ell), _ptr(means), _stream())
+                                   _ptr(x_out), _ptr(n_accept), _ptr(ell), _ptr(dist2), _ptr(means), _stream())
     _check(code, "spec_verify_fused")
-    return (x_out, n_accept) + ((ell,) if want_logratio else ()) + ((means,) if want_means else ())
+    return ((x_out, n_accept) + ((ell,) if want_logratio else ()) + ((means,) if want_means else ())
+            + ((dist2,) if want_dist2 else ()))
+
+
+def fit_lambda_profile(eps_delta, count=None, window=0):
+    """Relaxation table (Sec. 3.4) from per-transition prediction deviations: host-side fit inside the library.
+    eps_delta: [N] (index n-1 for transition n); count: [N] measurements per transition or None.  Returns fp32 [N]."""
+    e = np.ascontiguousarray(eps_delta, dtype=np.float64)
+    c = None if count is None else np.ascontiguousarray(count, dtype=np.int64)
+    out = np.empty(len(e), dtype=np.float32)
+    code = lib().free_fit_lambda_profile(e.ctypes.data_as(C.c_void_p), None if c is None else c.ctypes.data_as(C.c_void_p),
+                                         len(e), int(window), out.ctypes.data_as(C.c_void_p))
+    _check(code, "free_fit_lambda_profile")
+    return out
 
 
 class HostVerifier:
@@ -411,6 +429,20 @@ class Model:
                                 _ptr(_dev(labels, torch.int32)), float(cfg_scale), C.byref(sched.desc), _ptr(noise),
                                 _ptr(m_hat), _ptr(x_hat), _ptr(f_next), _ptr(ws), ws.numel(), _stream()), "draft_step")
         return m_hat, x_hat, f_next
+
+    def uncertainty_profile(self, x0, labels, sched: DeviceSchedule, K, cfg_scale, noise_target, noise_draft, uniforms, lam=None):
+        """The offline run of Sec. 3.4.  Returns (eps_delta [N], accept_prob [N], count [N]) as numpy arrays."""
+        B, N = x0.shape[0], sched.desc.N
+        _dev(x0, torch.float32); _dev(labels, torch.int32); _dev(noise_target, torch.float32)
+        prm = SpecParams(int(K), float(cfg_scale), None if lam is None else _dev(lam, torch.float32).data_ptr())
+        dev, acc, cnt = np.zeros(N), np.zeros(N), np.zeros(N, np.int64)
+        ws = self.workspace(B * max(int(K), 1))
+        _check(lib().free_uncertainty_profile(self.ctx, B, _ptr(x0), _ptr(labels), C.byref(sched.desc), C.byref(prm),
+                                              _ptr(noise_target), _ptr(noise_draft), _ptr(uniforms),
+                                              dev.ctypes.data_as(C.c_void_p), acc.ctypes.data_as(C.c_void_p),
+                                              cnt.ctypes.data_as(C.c_void_p), _ptr(ws), ws.numel(), _stream()),
+               "free_uncertainty_profile")
+        return dev, acc, cnt
 
     def sample_trajectory(self, x0, labels, sched: DeviceSchedule, K, cfg_scale, noise_target, noise_draft=None,
                           uniforms=None, lam=None):

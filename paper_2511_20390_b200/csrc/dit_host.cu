@@ -1,6 +1,7 @@
 // Host orchestration: context, workspace layout, the packed target pass, the drafter step and the
 // sampling loop (Algorithm 1).  Every numerical step is a kernel launch on the caller's stream.
 #include "internal.h"
+#include <math.h>
 #include <new>
 #include <string.h>
 #include <vector>
@@ -55,7 +56,7 @@ struct Workspace {
     float* head_out;
     // sampling loop
     float* fin_bias;
-    float *x_cur, *m_a, *pack_in, *x_draft, *m_draft, *sigma2_bk, *lam_bk, *u_bk, *cx_bk, *ce_bk;
+    float *x_cur, *m_a, *pack_in, *x_draft, *m_draft, *sigma2_bk, *lam_bk, *u_bk, *cx_bk, *ce_bk, *ell_bk, *d2_bk;
     void *feat0, *feat1;
     int32_t *cur_a, *nv, *n_acc, *t_step, *t_pack, *lab_pack, *t_draft, *act_draft, *active;
     size_t total;
@@ -103,6 +104,8 @@ Workspace plan(const free_ctx* c, int n, void* base) {
     w.u_bk = (float*)take(n * 4);
     w.cx_bk = (float*)take(n * 4);
     w.ce_bk = (float*)take(n * 4);
+    w.ell_bk = (float*)take(n * 4);
+    w.d2_bk = (float*)take(n * 4);
     w.feat0 = take(M * D * as);
     w.feat1 = take(M * D * as);
     for (int32_t** p : {&w.cur_a, &w.nv, &w.n_acc, &w.t_step, &w.t_pack, &w.lab_pack, &w.t_draft, &w.act_draft, &w.active})
@@ -572,7 +575,7 @@ int one_round(const free_ctx* c, const Workspace& w, const RoundIO& r, cudaStrea
         { Scope p(c, PC_VERIFY, (double)B * ((2.0 + G) * K + 2) * d * 4, s);
           FREE_TRY(spec_verify_fused_launch(B, K, d, G, r.cfg, w.head_out, w.pack_in, (long long)K * d,
                                             w.m_draft, w.x_draft, w.cx_bk, w.ce_bk, w.sigma2_bk, w.lam_bk, w.u_bk, w.nv, 0,
-                                            w.x_cur, w.n_acc, nullptr, nullptr, s)); }
+                                            w.x_cur, w.n_acc, w.ell_bk, w.d2_bk, nullptr, s)); }
     }
     Scope p(c, PC_CTRL, 0, s);
     cursor_update_kernel<<<(B + 127) / 128, 128, 0, s>>>(B, w.active, w.nv, w.n_acc, w.cur_a);
@@ -612,14 +615,18 @@ extern "C" int free_spec_round(free_ctx* c, int B, const float* x_cur, const int
     return FREE_OK;
 }
 
-extern "C" int sample_trajectory(free_ctx* c, int B, const float* x0, const int32_t* labels, const free_schedule* sch,
-                                 const free_spec_params* prm, const float* noise_target, const float* noise_draft,
-                                 const float* uniforms, float* x_final, free_traj_stats* stats,
-                                 void* ws, size_t ws_bytes, void* stream) {
-    if (!x0 || !labels || !prm || !noise_target || !x_final) return FREE_ERR_ARG;
-    FREE_TRY(check_round_args(c, B, prm->K, sch, ws, ws_bytes, noise_draft, uniforms));
+namespace {
+
+// Per-transition sums of what the verifier saw (Sec. 3.4: prediction deviation and acceptance probability).
+struct Diag { double* dev_sum; double* acc_sum; int64_t* count; };
+
+// Algorithm 1 for B samples: rounds until every cursor has passed N.  Host side of a round: cursors (loop control),
+// statistics and, when asked, the per-transition records of every examined draft.
+int run_trajectory(free_ctx* c, int B, const float* x0, const int32_t* labels, const free_schedule* sch,
+                   const free_spec_params* prm, const float* noise_target, const float* noise_draft,
+                   const float* uniforms, float* x_final, free_traj_stats* stats, const Diag* diag,
+                   void* ws, cudaStream_t s) {
     const int K = prm->K;
-    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     const Workspace w = plan(c, B * (K > 0 ? K : 1), ws);
     const int N = sch->N, d = c->d_latent;
     if (stats) memset(stats, 0, sizeof(*stats));
@@ -628,19 +635,28 @@ extern "C" int sample_trajectory(free_ctx* c, int B, const float* x0, const int3
     FREE_CUDA_TRY(cudaMemcpyAsync(w.x_cur, x0, (size_t)B * d * 4, cudaMemcpyDeviceToDevice, s));
     fill_i32_kernel<<<(B + 127) / 128, 128, 0, s>>>(B, 1, w.cur_a);
     FREE_TRY(free_check_launch());
-    std::vector<int32_t> h_a(B, 1), h_nv(B), h_acc(B), h_act(B);
+    std::vector<int32_t> h_a(B, 1), h_prev(B, 1), h_nv(B), h_acc(B), h_act(B);
+    std::vector<float> h_ell, h_d2, h_ce(N);
+    if (diag && K > 0) {
+        h_ell.resize((size_t)B * K); h_d2.resize((size_t)B * K);
+        FREE_CUDA_TRY(cudaMemcpyAsync(h_ce.data(), sch->coef_eps, (size_t)N * 4, cudaMemcpyDeviceToHost, s));
+    }
     RoundIO r{B, K, labels, sch, prm->cfg_scale, prm->lambda, noise_target, noise_draft, uniforms};
 
     for (long long round = 0; round < 2LL * N + 2; ++round) {
         bool any = false;
         for (int b = 0; b < B; ++b) any |= h_a[b] <= N;
         if (!any) break;
+        h_prev = h_a;
         FREE_TRY(one_round(c, w, r, s));
-        // host side of the round: cursors (loop control) and statistics
         FREE_CUDA_TRY(cudaMemcpyAsync(h_act.data(), w.active, B * 4, cudaMemcpyDeviceToHost, s));
         FREE_CUDA_TRY(cudaMemcpyAsync(h_nv.data(), w.nv, B * 4, cudaMemcpyDeviceToHost, s));
         if (K > 0) FREE_CUDA_TRY(cudaMemcpyAsync(h_acc.data(), w.n_acc, B * 4, cudaMemcpyDeviceToHost, s));
         FREE_CUDA_TRY(cudaMemcpyAsync(h_a.data(), w.cur_a, B * 4, cudaMemcpyDeviceToHost, s));
+        if (diag && K > 0) {
+            FREE_CUDA_TRY(cudaMemcpyAsync(h_ell.data(), w.ell_bk, (size_t)B * K * 4, cudaMemcpyDeviceToHost, s));
+            FREE_CUDA_TRY(cudaMemcpyAsync(h_d2.data(), w.d2_bk, (size_t)B * K * 4, cudaMemcpyDeviceToHost, s));
+        }
         uint32_t dev_err = 0;
         FREE_CUDA_TRY(cudaMemcpyAsync(&dev_err, w.err, 4, cudaMemcpyDeviceToHost, s));
         FREE_CUDA_TRY(cudaStreamSynchronize(s));
@@ -648,6 +664,18 @@ extern "C" int sample_trajectory(free_ctx* c, int B, const float* x0, const int3
         for (int b = 0; b < B; ++b) {
             if (!h_act[b]) continue;
             if (K > 0 && h_nv[b] > 0 && h_acc[b] < 0) return h_acc[b];
+            if (diag && K > 0 && h_nv[b] > 0) {
+                // examined drafts: the accepted ones and the rejected one; draft i verifies transition a + i + 1
+                const int seen = h_acc[b] < h_nv[b] ? h_acc[b] + 1 : h_nv[b];
+                for (int i = 0; i < seen; ++i) {
+                    const int t = h_prev[b] + i + 1;
+                    const double ell = (double)h_ell[(size_t)b * K + i], d2 = (double)h_d2[(size_t)b * K + i];
+                    const double ce = (double)h_ce[N - t];
+                    diag->dev_sum[t - 1] += ce != 0.0 ? sqrt(d2) / fabs(ce) : 0.0;
+                    diag->acc_sum[t - 1] += ell < 0.0 ? exp(ell) : 1.0;
+                    diag->count[t - 1] += 1;
+                }
+            }
             if (!stats) continue;
             stats->target_calls += 1;
             if (h_nv[b] > 0) {
@@ -660,9 +688,38 @@ extern "C" int sample_trajectory(free_ctx* c, int B, const float* x0, const int3
         }
         if (stats) stats->rounds += 1;
     }
-    FREE_CUDA_TRY(cudaMemcpyAsync(x_final, w.x_cur, (size_t)B * d * 4, cudaMemcpyDeviceToDevice, s));
+    if (x_final) FREE_CUDA_TRY(cudaMemcpyAsync(x_final, w.x_cur, (size_t)B * d * 4, cudaMemcpyDeviceToDevice, s));
     FREE_CUDA_TRY(cudaStreamSynchronize(s));
     if (stats && stats->target_calls > 0) stats->parallel_efficiency = (double)B * N / (double)stats->target_calls;
+    return FREE_OK;
+}
+
+}  // namespace
+
+extern "C" int sample_trajectory(free_ctx* c, int B, const float* x0, const int32_t* labels, const free_schedule* sch,
+                                 const free_spec_params* prm, const float* noise_target, const float* noise_draft,
+                                 const float* uniforms, float* x_final, free_traj_stats* stats,
+                                 void* ws, size_t ws_bytes, void* stream) {
+    if (!x0 || !labels || !prm || !noise_target || !x_final) return FREE_ERR_ARG;
+    FREE_TRY(check_round_args(c, B, prm->K, sch, ws, ws_bytes, noise_draft, uniforms));
+    return run_trajectory(c, B, x0, labels, sch, prm, noise_target, noise_draft, uniforms, x_final, stats, nullptr, ws,
+                          reinterpret_cast<cudaStream_t>(stream));
+}
+
+extern "C" int free_uncertainty_profile(free_ctx* c, int B, const float* x0, const int32_t* labels, const free_schedule* sch,
+                                        const free_spec_params* prm, const float* noise_target, const float* noise_draft,
+                                        const float* uniforms, double* eps_delta, double* accept_prob, int64_t* count,
+                                        void* ws, size_t ws_bytes, void* stream) {
+    if (!x0 || !labels || !prm || !noise_target || !eps_delta || !accept_prob || !count) return FREE_ERR_ARG;
+    if (prm->K < 1) return FREE_ERR_SHAPE;
+    FREE_TRY(check_round_args(c, B, prm->K, sch, ws, ws_bytes, noise_draft, uniforms));
+    const int N = sch->N;
+    for (int n = 0; n < N; ++n) { eps_delta[n] = 0.0; accept_prob[n] = 0.0; count[n] = 0; }
+    const Diag diag{eps_delta, accept_prob, count};
+    FREE_TRY(run_trajectory(c, B, x0, labels, sch, prm, noise_target, noise_draft, uniforms, nullptr, nullptr, &diag, ws,
+                            reinterpret_cast<cudaStream_t>(stream)));
+    for (int n = 0; n < N; ++n)
+        if (count[n] > 0) { eps_delta[n] /= (double)count[n]; accept_prob[n] /= (double)count[n]; }
     return FREE_OK;
 }
 

@@ -87,4 +87,4 @@ int spec_verify_fused_launch(int B, int K, long long d, int G, float cfg_scale,
                              const float* eps, const float* x_first, long long x_first_stride,
                              const float* m_draft, const float* x_draft, const float* coef_x, const float* coef_eps,
                              const float* sigma2, const float* lambda, const float* u, const int32_t* n_valid, int chunk,
-                             float* x_out, int32_t* n_accept, float* logratio_out, float* means_out, cudaStream_t s);
+                             float* x_out, int32_t* n_accept, float* logratio_out, float* dist2_out, float* means_out, cudaStream_t s);

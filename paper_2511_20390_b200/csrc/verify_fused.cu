@@ -29,7 +29,7 @@ struct FusedArgs {
     const float* x_first; long long x_first_stride;
     const float *mh, *xh, *coef_x, *coef_eps, *sigma2, *lambda, *u;
     const int32_t* n_valid;
-    float* x_out; int32_t* n_accept; float* logratio; float* means_out;
+    float* x_out; int32_t* n_accept; float* logratio; float* dist2; float* means_out;
 };
 
 struct Row {                      // operands of draft k of this sample
@@ -180,6 +180,7 @@ __global__ void __launch_bounds__(kThreads, 4) spec_verify_fused_kernel(FusedArg
     if (rank == 0) {
         if (tid == 0) a.n_accept[b] = err ? FREE_ERR_SIGMA : j;
         if (a.logratio && tid < K) a.logratio[(size_t)b * K + tid] = tid < examined ? (float)ell_s[tid] : nanf("");
+        if (a.dist2 && tid < K) a.dist2[(size_t)b * K + tid] = tid < examined ? (float)tot[tid][0] : nanf("");
     }
     if (err || nv == 0) return;
 
@@ -250,7 +251,7 @@ int spec_verify_fused_launch(int B, int K, long long d, int G, float cfg_scale,
                              const float* eps, const float* x_first, long long x_first_stride,
                              const float* m_draft, const float* x_draft, const float* coef_x, const float* coef_eps,
                              const float* sigma2, const float* lambda, const float* u, const int32_t* n_valid, int chunk,
-                             float* x_out, int32_t* n_accept, float* logratio_out, float* means_out, cudaStream_t s) {
+                             float* x_out, int32_t* n_accept, float* logratio_out, float* dist2_out, float* means_out, cudaStream_t s) {
     if (B < 0 || !eps || !x_first || !m_draft || !x_draft || !coef_x || !coef_eps || !sigma2 || !u || !x_out || !n_accept)
         return FREE_ERR_ARG;
     if (G != 1 && G != 2) return FREE_ERR_ARG;
@@ -261,7 +262,7 @@ int spec_verify_fused_launch(int B, int K, long long d, int G, float cfg_scale,
         !free_aligned16(x_out) || !free_aligned16(means_out))
         return FREE_ERR_ALIGN;
     FusedArgs a{B, K, G, chunk, d, cfg_scale, eps, x_first, x_first_stride, m_draft, x_draft, coef_x, coef_eps,
-                sigma2, lambda, u, n_valid, x_out, n_accept, logratio_out, means_out};
+                sigma2, lambda, u, n_valid, x_out, n_accept, logratio_out, dist2_out, means_out};
     const bool vec = (d % 4) == 0 && (x_first_stride % 4) == 0;      // every row stays 16-byte aligned only then
     if (!vec) return d >= 4096 ? launch_g<4, false>(a, s) : launch_g<1, false>(a, s);
     int dev = 0, sms = 148;
@@ -281,8 +282,8 @@ extern "C" int spec_verify_fused(int B, int K, int64_t d, int G, float cfg_scale
                                  const float* eps, const float* x_first, const float* m_draft, const float* x_draft,
                                  const float* coef_x, const float* coef_eps, const float* sigma2, const float* lambda,
                                  const float* u, const int32_t* n_valid, int chunk,
-                                 float* x_out, int32_t* n_accept, float* logratio_out, float* means_out, void* stream) {
+                                 float* x_out, int32_t* n_accept, float* logratio_out, float* dist2_out, float* means_out, void* stream) {
     return spec_verify_fused_launch(B, K, (long long)d, G, cfg_scale, eps, x_first, (long long)d, m_draft, x_draft, coef_x, coef_eps,
-                                    sigma2, lambda, u, n_valid, chunk, x_out, n_accept, logratio_out, means_out,
+                                    sigma2, lambda, u, n_valid, chunk, x_out, n_accept, logratio_out, dist2_out, means_out,
                                     reinterpret_cast<cudaStream_t>(stream));
 }

@@ -98,7 +98,7 @@ def test_fused_verifier_stays_in_bounds():
     cu = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(torch.float32).cuda()
     one = torch.ones(B, K, device="cuda", dtype=torch.float32)
     x_out, means, n_acc = Guarded(B * d * 4, torch.float32), Guarded(B * K * d * 4, torch.float32), Guarded(B * 4, torch.int32)
-    ell = Guarded(B * K * 4, torch.float32)
+    ell, d2 = Guarded(B * K * 4, torch.float32), Guarded(B * K * 4, torch.float32)
     L = free.lib()
     st = torch.cuda.current_stream().cuda_stream
     ts = [cu(eps), cu(x_first), cu(mh), cu(xh)]
@@ -106,7 +106,7 @@ def test_fused_verifier_stays_in_bounds():
     for chunk in (0, 2):
         rc = L.spec_verify_fused(B, K, d, G, 4.0, ts[0].data_ptr(), ts[1].data_ptr(), ts[2].data_ptr(), ts[3].data_ptr(),
                                  one.data_ptr(), ce.data_ptr(), s2.data_ptr(), None, uu.data_ptr(), None, chunk,
-                                 x_out.t.data_ptr(), n_acc.t.data_ptr(), ell.t.data_ptr(), means.t.data_ptr(), st)
+                                 x_out.t.data_ptr(), n_acc.t.data_ptr(), ell.t.data_ptr(), d2.t.data_ptr(), means.t.data_ptr(), st)
         assert rc == 0
         torch.cuda.synchronize()
-        assert x_out.intact() and means.intact() and n_acc.intact() and ell.intact()
+        assert x_out.intact() and means.intact() and n_acc.intact() and ell.intact() and d2.intact()

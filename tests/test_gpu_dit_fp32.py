@@ -153,3 +153,40 @@ def test_trajectory_tiny_matches_oracle(free, K, cfg, relaxed):
         assert acc > 5 and rej > 5
     if K == 0:
         assert st["target_calls"] == B * N and st["draft_calls"] == 0
+
+
+@pytest.mark.parametrize("K,cfg", [(4, 0.0), (3, 4.0)])
+def test_uncertainty_profile_tiny_matches_oracle(free, K, cfg):
+    """The offline run of Sec. 3.4 (per-transition prediction deviation and acceptance probability of every examined
+    draft) against the oracle's recorder on the same trajectories, and the relaxation table fitted from it."""
+    from oracle import relax as orelax
+    sh, w, wd, model = _tiny_model(free)
+    N, B = 50, 2
+    sc = osched.make("linear", N)
+    dsched = free.DeviceSchedule(free.linear_schedule(N))
+    shape = (sh.C, sh.H, sh.W)
+    x0 = synth.normal(6, 1, (B,) + shape)
+    zt, zd = synth.normal(6, 2, (B, N) + shape), synth.normal(6, 3, (B, N) + shape)
+    u = synth.uniform01(6, 4, (B, N))
+    labels = np.array([2, 8], np.int32)
+    dev, acc, cnt = model.uncertainty_profile(cu(x0), cu(labels, torch.int32), dsched, K, cfg, cu(zt), cu(zd), cu(u))
+    rec = orelax.Recorder(N, sc.coef_eps)
+    for b in range(B):
+        def target(x, s, b=b):
+            m, _, f = odit.verify_pass(w, sh, sc, x[None], [s], [int(labels[b])], cfg)
+            return m[0], f[0]
+
+        def draft(xp, f, s, b=b):
+            m, _, fn = odrafter.guided_step(w, wd, sh, sc, xp, f, s, int(labels[b]), cfg)
+            return m, fn
+        trace = []
+        otraj.sample(x0[b], N, K, target, draft, sc.sigma2, zt[b], zd[b], u[b], trace=trace, observe=rec)
+        assert all(abs(ell - np.log(u[b, t - 1])) > 1e-3 for t, ok, ell in trace if ell < 0)
+    dev_o, acc_o, cnt_o = rec.profile()
+    assert np.array_equal(cnt, cnt_o) and cnt.sum() > 10 and cnt[0] == 0 and cnt[-1] == 0
+    seen = cnt > 0
+    assert np.allclose(dev[seen], dev_o[seen], rtol=1e-3) and np.all(dev[~seen] == 0)
+    assert np.allclose(acc[seen], acc_o[seen], atol=2e-3)
+    lam = free.fit_lambda_profile(dev, cnt, 2)
+    assert np.allclose(lam, orelax.lambda_profile(dev_o, cnt_o, 2), rtol=2e-3)
+    assert lam[0] == 1.0 and np.all(np.diff(lam) <= 0) and np.all(lam > 0)

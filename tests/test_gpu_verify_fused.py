@@ -38,6 +38,14 @@ def _run(i, w_cfg, lam=None, n_valid=None, chunk=0):
     return x.cpu().numpy(), n.cpu().numpy(), ell.cpu().numpy(), means.cpu().numpy()
 
 
+def _dist2(i, w_cfg, chunk=0):
+    import paper_2511_20390_b200 as free
+    out = free.spec_verify_fused(cu(i["eps"]), cu(i["x_first"]), cu(i["m_hat"]), cu(i["x_hat"]), cu(i["cx"]), cu(i["ce"]),
+                                 cu(i["s2"]), cu(i["u"]), w_cfg, chunk=chunk, want_logratio=True, want_dist2=True)
+    torch.cuda.synchronize()
+    return out[1].cpu().numpy(), out[2].cpu().numpy(), out[3].cpu().numpy()
+
+
 def _compare(i, w_cfg, lam=None, n_valid=None, chunk=0):
     B, K = i["u"].shape
     x, n, ell, means = _run(i, w_cfg, lam, n_valid, chunk)
@@ -115,6 +123,19 @@ def test_mixed_decisions_relaxed_ragged_and_early_exit():
     assert np.array_equal(n_rc, n_r)
 
 
+def test_mean_distance_output():
+    # |m_hat - m|^2 per examined draft, against the oracle's means; NaN exactly where the log-ratio is NaN
+    shape, G, B, K = (4, 32, 32), 2, 6, 8
+    i = _inputs(31, B, K, shape, G, s_rel=0.6)
+    mo = np.stack([overify.means_from_stream_eps(i["eps"][b], i["x_first"][b], i["x_hat"][b], i["cx"][b], i["ce"][b], 1.5) for b in range(B)])
+    ref = ((i["m_hat"].astype(np.float64) - mo) ** 2).sum(axis=(2, 3, 4))
+    for chunk in (0, 2):
+        n, ell, d2 = _dist2(i, 1.5, chunk)
+        seen = ~np.isnan(ell)
+        assert np.array_equal(np.isnan(d2), ~seen) and (chunk > 0 or seen.all())
+        assert np.allclose(d2[seen], ref[seen], rtol=1e-6)
+
+
 def test_degenerate_cases():
     shape, G, B, K = (4, 16, 16), 2, 4, 3
     i = _inputs(9, B, K, shape, G, s_rel=30.0)
@@ -147,7 +168,7 @@ def test_argument_errors():
     with pytest.raises(free.FreeError):                     # three streams
         _run(dict(i, eps=np.concatenate([i["eps"], i["eps"][:, :, :1]], axis=2)), 4.0)
     L = free.lib()
-    assert L.spec_verify_fused(1, 0, 16, 1, 1.0, *([None] * 10), 0, *([None] * 5)) != 0
+    assert L.spec_verify_fused(1, 0, 16, 1, 1.0, *([None] * 10), 0, *([None] * 6)) != 0
 
 
 def test_full_size_point_sampled_against_oracle():
