@@ -190,3 +190,26 @@ def test_uncertainty_profile_tiny_matches_oracle(free, K, cfg):
     lam = free.fit_lambda_profile(dev, cnt, 2)
     assert np.allclose(lam, orelax.lambda_profile(dev_o, cnt_o, 2), rtol=2e-3)
     assert lam[0] == 1.0 and np.all(np.diff(lam) <= 0) and np.all(lam > 0)
+
+
+@pytest.mark.parametrize("kw", [{"stochasticity": 0.7}, {"variance": "beta"}, {"variance": 0.5}])
+def test_trajectory_with_other_variance_schedules(free, kw):
+    """Other fixed-variance schedules and the stochasticity family (Appendices "Variance Setting" / "Stochasticity
+    Hyperparameter") are tables to the kernels: the whole loop against the oracle with the oracle's own tables."""
+    sh, w, wd, model = _tiny_model(free)
+    N, B, K, cfg = 50, 2, 4, 0.0
+    sc = osched.make("linear", N, **kw)
+    dsched = free.DeviceSchedule(free.linear_schedule(N, **kw))
+    shape = (sh.C, sh.H, sh.W)
+    x0 = synth.normal(14, 1, (B,) + shape)
+    zt, zd = synth.normal(14, 2, (B, N) + shape), synth.normal(14, 3, (B, N) + shape)
+    u = synth.uniform01(14, 4, (B, N))
+    labels = np.array([1, 6], np.int32)
+    xf, st = model.sample_trajectory(cu(x0), cu(labels, torch.int32), dsched, K, cfg, cu(zt), cu(zd), cu(u))
+    acc = rej = 0
+    for b in range(B):
+        xo, so, trace = _oracle_traj(sh, w, wd, sc, N, K, cfg, x0[b], int(labels[b]), zt[b], zd[b], u[b])
+        assert all(abs(ell - np.log(u[b, t - 1])) > 1e-3 for t, ok, ell in trace if ell < 0)
+        assert nerr(xf[b], xo) < 5 * TOL
+        acc += so["accepted"]; rej += so["rejected"]
+    assert st["accepted"] == acc and st["rejected"] == rej and acc + rej > 10

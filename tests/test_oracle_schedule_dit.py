@@ -51,6 +51,68 @@ def test_mean_is_the_posterior_mean_for_the_true_noise(kind, N):
     assert np.allclose(sc.mean(x0, 0 * x0, 3), x0 / np.sqrt(sc.alphas[3]))
 
 
+def _variance_after_chain(sc, s0_sq):
+    """Variance of x_0 when data ~ N(0, s0_sq) and the chain runs with the EXACT noise prediction of that Gaussian
+    (eps*(x, s) = sqrt(1 - abar_s) x / v_s, v_s = abar_s s0_sq + 1 - abar_s).  Also returns the largest relative
+    gap to the forward marginals on the way."""
+    v = sc.abar[-1] * s0_sq + 1.0 - sc.abar[-1]
+    worst = 0.0
+    for s in range(sc.N - 1, -1, -1):
+        v_s = sc.abar[s] * s0_sq + 1.0 - sc.abar[s]
+        gain = sc.coef_x[s] - sc.coef_eps[s] * np.sqrt(1.0 - sc.abar[s]) / v_s
+        v = gain * gain * v + sc.sigma2[s]
+        target = (sc.abar[s - 1] * s0_sq + 1.0 - sc.abar[s - 1]) if s > 0 else s0_sq
+        worst = max(worst, abs(v / target - 1.0))
+    return v, worst
+
+
+@pytest.mark.parametrize("s0_sq", [0.25, 1.0, 4.0])
+@pytest.mark.parametrize("eps", [0.0, 0.5, 1.0, 1.5])
+def test_stochasticity_family_shares_the_marginals(eps, s0_sq):
+    # Appendix "Stochasticity Hyperparameter": with the exact score every member of the family has the forward marginals
+    # (up to the discretisation error of 1000 Euler-Maruyama steps)
+    sc = schedule.Schedule(schedule.linear_betas(1000), stochasticity=eps)
+    v, worst = _variance_after_chain(sc, s0_sq)
+    assert abs(v / s0_sq - 1.0) < 0.03 and worst < 0.03
+
+
+def test_stochasticity_special_members():
+    b = schedule.linear_betas(100)
+    ode = schedule.Schedule(b, stochasticity=0.0)
+    assert np.all(ode.sigma2 == 0) and np.allclose(ode.coef_eps, 0.5 * b / np.sqrt(1 - ode.abar))      # probability-flow ODE
+    sde, ddpm = schedule.Schedule(b, stochasticity=1.0), schedule.Schedule(b, variance="beta")
+    # eps = 1 is the first-order (in beta) form of the DDPM step with sigma^2 = beta
+    assert np.all(np.abs(sde.coef_x - ddpm.coef_x) <= b ** 2)
+    assert np.allclose(sde.coef_eps, ddpm.coef_eps * np.sqrt(ddpm.alphas), rtol=1e-12)
+    assert np.array_equal(sde.sigma2, ddpm.sigma2)
+    two = schedule.Schedule(b, stochasticity=2.0)
+    assert np.allclose(two.sigma2, 4 * sde.sigma2) and np.allclose(two.coef_eps, 2.5 * sde.coef_eps)
+
+
+@pytest.mark.parametrize("variance", ["posterior", "beta", 0.3])
+def test_fixed_variance_choices(variance):
+    b = schedule.linear_betas(1000)
+    sc, post, beta = schedule.Schedule(b, variance=variance), schedule.Schedule(b), schedule.Schedule(b, variance="beta")
+    assert np.array_equal(sc.coef_x, post.coef_x) and np.array_equal(sc.coef_eps, post.coef_eps)     # only sigma changes
+    assert sc.sigma2[0] == 0.0 and np.all(sc.sigma2[1:] >= post.sigma2[1:] * (1 - 1e-12)) and np.all(sc.sigma2[1:] <= b[1:] * (1 + 1e-12))
+    if variance == 0.3:
+        assert np.allclose(np.log(sc.sigma2[1:]), 0.3 * np.log(b[1:]) + 0.7 * np.log(post.sigma2[1:]))
+        assert np.allclose(schedule.Schedule(b, variance=0.0).sigma2, post.sigma2) and np.allclose(schedule.Schedule(b, variance=1.0).sigma2[1:], b[1:])
+    # any sigma between the two extremes keeps the marginals of unit-variance data (where beta is exact) within a few percent
+    v, _ = _variance_after_chain(sc, 1.0)
+    assert abs(v - 1.0) < 0.03
+
+
+def test_library_schedule_tables_match_oracle():
+    from paper_2511_20390_b200 import schedule as product
+    for kw in ({}, {"variance": "beta"}, {"variance": 0.4}, {"stochasticity": 0.7}, {"stochasticity": 0.0}):
+        for name, N in (("linear", 50), ("respaced", 250)):
+            o = schedule.make(name, N, **kw)
+            t = getattr(product, name + "_schedule")(N, **kw)
+            for key in ("coef_x", "coef_eps", "sigma2", "t_embed_value"):
+                assert np.allclose(t[key], getattr(o, key), rtol=1e-13, atol=0), (kw, name, key)
+
+
 def test_respaced_keeps_abar_of_the_full_schedule():
     b, idx = schedule.respaced_betas(250)
     full = np.cumprod(1.0 - schedule.linear_betas(1000))
