@@ -39,4 +39,4 @@ def test_total_is_the_weighted_sum():
     ln, lf, ls, tot = losses.free_loss(e1, e2, p, r, 0.5, 0.01, beta=0.7)
     assert np.isclose(tot, ln + 0.5 * lf + 0.01 * ls) and ln > 0 and 0 < lf < 2 and ls > 0
     # the noise term and the feature terms do not mix
-    assert losses.free_loss(e1, e1, p, p, 0.5, 0.01)[3] < 1e-12
+    assert losses.free_loss(e1, e1, p, p, 0.5, 0.01, eps_cos=0.0)[3] < 1e-12
