@@ -1,6 +1,6 @@
 """Benchmark of the packed parallel-verification path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload round|verifier|verifier_fused|trajectory] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload round|verifier|verifier_fused|drafter_loss|trajectory] [--impl reference]
 
 One JSON line on stdout (rank 0).  A "step" is one pass of the hot path over one batch of synthetic
 input resident in HBM; `e2e` repeats it from pinned HOST buffers with the copies inside the timed
@@ -242,7 +242,64 @@ class FusedVerifierWorkload:
         return nb * self.bytes_per_step / self.B / 1e9 / dt, f"{nb} of {self.B} samples of the same batch, full K"
 
 
+class DrafterLossWorkload:
+    """The drafter's training objectives (Sec. 3.2) on DiT-XL/2 512^2 shapes: per sample a bf16 top-block feature pair
+    [1024, 1152] and an fp32 noise pair [4, 64, 64]; 256 samples per step (1.24 GB, larger than L2)."""
+    name = "drafter loss, 256 samples, features [1024, 1152] bf16, noise 4x64x64"
+    metric, unit, dtype = "loss reduction HBM GB/s", "GB/s", "f32"
+
+    def __init__(self, batch, rank):
+        import torch
+        import paper_2511_20390_b200 as free
+        self.torch, self.free = torch, free
+        self.n, self.n_tok, self.D, self.d_eps = (batch or 256), 1024, 1152, 16384
+        g = torch.Generator(device="cuda"); g.manual_seed(3000 + rank)
+        mk = lambda *s: torch.randn(*s, generator=g, device="cuda", dtype=torch.float32)
+        self.f_ref = mk(self.n, self.n_tok, self.D).bfloat16()
+        self.f_pred = (self.f_ref.float() + 0.3 * mk(self.n, self.n_tok, self.D)).bfloat16()
+        self.e_ref = mk(self.n, self.d_eps)
+        self.e_pred = self.e_ref + 0.1 * mk(self.n, self.d_eps)
+        self.out = torch.empty(4, dtype=torch.float64, device="cuda")
+        self.bytes_per_step = 2 * self.n * self.n_tok * self.D * 2 + 2 * self.n * self.d_eps * 4
+        self.units_per_step = self.bytes_per_step / 1e9
+        self.launches_per_step = 2
+        self.pinned = None
+        self.config = {"workload": self.name, "samples": self.n, "cache": "inputs larger than L2 (1.24 GB per step)"}
+
+    def step(self):
+        self.free.drafter_loss(self.e_pred, self.e_ref, self.f_pred, self.f_ref, 0.5, 0.01, out=self.out)
+
+    def host_step(self):
+        torch = self.torch
+        if self.pinned is None:
+            self.pinned = [t.cpu().pin_memory() for t in (self.e_pred, self.e_ref, self.f_pred, self.f_ref)]
+            self.stage = [torch.empty_like(t, device="cuda") for t in self.pinned]
+            self.h_out = torch.empty(4, dtype=torch.float64, pin_memory=True)
+        for d, h in zip(self.stage, self.pinned):
+            d.copy_(h, non_blocking=True)
+        self.free.drafter_loss(*self.stage, 0.5, 0.01, out=self.out)
+        self.h_out.copy_(self.out, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        return sum(t.numel() * t.element_size() for t in self.pinned), 32
+
+    def roofline(self, ms_per_step, peaks):
+        ach = self.bytes_per_step / 1e9 / (ms_per_step / 1e3)
+        return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+                "traffic": None, "kernel": "loss_partial_kernel", "peak_source": peaks["source"]}
+
+    def oracle_sample(self):
+        from oracle import losses as ol
+        nb = 8
+        a = [t[:nb].float().cpu().numpy() for t in (self.e_pred, self.e_ref, self.f_pred, self.f_ref)]
+        t0 = time.perf_counter()
+        ol.free_loss(*a, 0.5, 0.01)
+        dt = time.perf_counter() - t0
+        return nb * self.bytes_per_step / self.n / 1e9 / dt, f"{nb} of {self.n} samples of the same batch"
+
+
 def make_workload(name, batch, rank, chunk=0):
+    if name == "drafter_loss":
+        return DrafterLossWorkload(batch, rank)
     if name in ("verifier",):
         return VerifierWorkload(batch, rank)
     if name == "verifier_fused":

@@ -315,6 +315,26 @@ typedef struct free_prof_entry {
 int free_profile_begin(free_ctx* ctx);
 int free_profile_end(free_ctx* ctx, free_prof_entry* out, int max_entries, int* n_entries);
 
+/*
+ * free_drafter_loss -- the drafter's training objectives (Sec. 3.2), forward values, as one fused reduction:
+ *   L_noise  = mean over all elements of (eps_pred - eps_ref)^2                                   (Eq. mse)
+ *   L_feat   = mean over sequences and tokens of 1 - <p, r> / (|p| |r| + eps_cos)                 (Eq. cos)
+ *   L_smooth = mean over sequences, tokens and channels of phi_beta(p - r)                        (Eqs. smooth, huber)
+ *   L_total  = L_noise + lambda_f L_feat + lambda_s L_smooth                                      (Eq. free_loss)
+ *   dtype            FREE_FP32 or FREE_BF16: type of the features
+ *   eps_pred, eps_ref   DEVICE fp32 [n_seq, d_eps]
+ *   f_pred, f_ref       DEVICE `dtype` [n_seq, n_tok, D] (top-block features)
+ *   beta > 0, eps_cos >= 0
+ *   out              DEVICE double [4]: L_noise, L_feat, L_smooth, L_total
+ *   ws               DEVICE, >= free_drafter_loss_workspace_bytes(): per-CTA partial sums (added in a fixed order)
+ * Asynchronous.  Errors: ARG, SHAPE, WORKSPACE, ALIGN, CUDA.
+ */
+size_t free_drafter_loss_workspace_bytes(void);
+int free_drafter_loss(int dtype, int n_seq, int n_tok, int D, int64_t d_eps,
+                      const float* eps_pred, const float* eps_ref, const void* f_pred, const void* f_ref,
+                      float lambda_f, float lambda_s, float beta, float eps_cos,
+                      double* out, void* ws, size_t ws_bytes, void* stream);
+
 /* ------------------------------------------------------------------------------------------------
  * Building blocks, exported so that each kernel can be checked against the CPU oracle on its own.
  * They are the same kernels the calls above launch.

@@ -86,6 +86,9 @@ _SIGNATURES = {
                                            C.POINTER(SpecParams), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "free_fit_lambda_profile": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p]),
+    "free_drafter_loss_workspace_bytes": (C.c_size_t, []),
+    "free_drafter_loss": (C.c_int, [C.c_int] * 4 + [C.c_int64] + [C.c_void_p] * 4 + [C.c_float] * 4 +
+                          [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "free_profile_begin": (C.c_int, [C.c_void_p]),
     "free_profile_end": (C.c_int, [C.c_void_p, C.POINTER(ProfEntry), C.c_int, C.POINTER(C.c_int)]),
     "free_op_linear_workspace_bytes": (C.c_size_t, []),
@@ -182,6 +185,27 @@ def spec_verify_fused(eps, x_first, m_hat, x_hat, coef_x, coef_eps, sigma2, u, c
     _check(code, "spec_verify_fused")
     return ((x_out, n_accept) + ((ell,) if want_logratio else ()) + ((means,) if want_means else ())
             + ((dist2,) if want_dist2 else ()))
+
+
+_LOSS_WS = {}
+
+
+def drafter_loss(eps_pred, eps_ref, f_pred, f_ref, lambda_f, lambda_s, beta=1.0, eps_cos=1e-8, out=None):
+    """Drafter training objectives (Sec. 3.2) in one fused reduction.  eps_*: CUDA fp32 [n, d...]; f_*: CUDA fp32 or
+    bf16 [n, n_tok, D].  Returns a CUDA float64 tensor (L_noise, L_feat, L_smooth, L_total)."""
+    n, n_tok, D = f_pred.shape
+    _dev(eps_pred, torch.float32); _dev(eps_ref, torch.float32); _dev(f_ref, f_pred.dtype)
+    dtype = {torch.float32: FREE_FP32, torch.bfloat16: FREE_BF16}[f_pred.dtype]
+    _dev(f_pred, f_pred.dtype)
+    if out is None:
+        out = torch.empty(4, dtype=torch.float64, device=f_pred.device)
+    ws = _LOSS_WS.get(f_pred.device)
+    if ws is None:
+        ws = _LOSS_WS[f_pred.device] = torch.empty(lib().free_drafter_loss_workspace_bytes(), dtype=torch.uint8, device=f_pred.device)
+    _check(lib().free_drafter_loss(dtype, n, n_tok, D, eps_pred.numel() // n, _ptr(eps_pred), _ptr(eps_ref), _ptr(f_pred), _ptr(f_ref),
+                                   float(lambda_f), float(lambda_s), float(beta), float(eps_cos), _ptr(out), _ptr(ws), ws.numel(),
+                                   _stream()), "free_drafter_loss")
+    return out
 
 
 def fit_lambda_profile(eps_delta, count=None, window=0):
