@@ -231,7 +231,7 @@ class OpsWorkload:
 
 def run_trajectory(args):
     """`bench.py --workload trajectory`: whole sampling trajectories (Algorithm 1 end to end through sample_trajectory)
-    on the DiT-XL/2-shaped 512^2 model, 250 transitions, guidance, batch B: images per second for the two bounding
+    on the DiT-XL/2-shaped 512^2 (or, with --res 256, 256^2) model, 250 transitions, guidance, batch B: images per second for the two bounding
     acceptance regimes (u = 0: every draft accepted; u = 1: a draft is accepted only if its log-ratio is >= 0, which a
     random-init drafter almost never reaches), for seeded uniforms, and for the plain sequential sampler (K = 0) on
     the same GPU.  One trajectory per regime after one warm-up trajectory; device time by CUDA events."""
@@ -240,7 +240,8 @@ def run_trajectory(args):
     import synth
     import paper_2511_20390_b200 as free
     torch.cuda.set_device(0)
-    sh = synth.DIT_XL2_512
+    res = getattr(args, "res", 512)
+    sh = synth.DIT_XL2_256 if res == 256 else synth.DIT_XL2_512
     B = args.batch or 16
     model = free.Model.random(sh, 1234, dtype="bf16", with_drafter=True)
     sched = free.DeviceSchedule(free.respaced_schedule(N_SCHED))
@@ -270,7 +271,7 @@ def run_trajectory(args):
                      "parallel_efficiency": st["parallel_efficiency"]}
     line = {"metric": "images/s", "value": out["all_accepted"]["images_per_s"], "unit": "images/s", "n_gpus": 1,
             "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": f"sample_trajectory, DiT-XL/2-shaped 512^2, {N_SCHED} transitions, K={K_DRAFTS}, cfg {CFG}, batch {B}; "
+            "config": {"workload": f"sample_trajectory, DiT-XL/2-shaped {res}^2, {N_SCHED} transitions, K={K_DRAFTS}, cfg {CFG}, batch {B}; "
                                    "value = the all-accepted regime"},
             "regimes": out}
     print(json.dumps(line))
