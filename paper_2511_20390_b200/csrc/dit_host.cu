@@ -300,16 +300,17 @@ int drafter_pass(const free_ctx* c, const Workspace& w, int n_states, float cfg,
     FREE_TRY(run_cond(c, w, st, n_states, G, io.t_idx, io.labels, sch, s));
     { Scope p(c, PC_EMBED, (double)M * D * as, s);
       FREE_TRY(patch_embed(m.dtype, n_states, G, m.C, m.H, m.W, m.patch, D, io.x_in, io.x_stride, m.pe_w, m.pe_b, m.pos, w.emb, s)); }
-    Scope* fc = new Scope(c, PC_DRAFT_FC, 2.0 * M * D * 2 * D, s);
-    // g = W_fc [embed || f] + b  as two accumulating GEMMs over the two halves of W_fc (row stride 2D)
-    LinearArgs a; a.err = w.err;
-    a.M = M; a.N = D; a.K = D; a.A = w.emb; a.W = c->dr.fc_w; a.ldw = 2 * D; a.bias = c->dr.fc_b;
-    a.epi = EPI_BIAS; a.out_dtype = FREE_FP32; a.out = w.x;
-    { const int r1 = lin(c, a, s); if (r1 != FREE_OK) { delete fc; return r1; } }
-    a = LinearArgs(); a.err = w.err;
-    a.M = M; a.N = D; a.K = D; a.A = f_prev; a.W = (const char*)c->dr.fc_w + (size_t)D * as; a.ldw = 2 * D;
-    a.epi = EPI_GATE_RESIDUAL; a.resid = w.x; a.gate = nullptr; a.rows_per_seq = c->n_tok;
-    { const int r2 = lin(c, a, s); delete fc; FREE_TRY(r2); }
+    {   // g = W_fc [embed || f] + b  as two accumulating GEMMs over the two halves of W_fc (row stride 2D)
+        Scope fc(c, PC_DRAFT_FC, 2.0 * M * D * 2 * D, s);
+        LinearArgs a; a.err = w.err;
+        a.M = M; a.N = D; a.K = D; a.A = w.emb; a.W = c->dr.fc_w; a.ldw = 2 * D; a.bias = c->dr.fc_b;
+        a.epi = EPI_BIAS; a.out_dtype = FREE_FP32; a.out = w.x;
+        FREE_TRY(lin(c, a, s));
+        a = LinearArgs(); a.err = w.err;
+        a.M = M; a.N = D; a.K = D; a.A = f_prev; a.W = (const char*)c->dr.fc_w + (size_t)D * as; a.ldw = 2 * D;
+        a.epi = EPI_GATE_RESIDUAL; a.resid = w.x; a.gate = nullptr; a.rows_per_seq = c->n_tok;
+        FREE_TRY(lin(c, a, s));
+    }
     FREE_TRY(run_blocks(c, w, st, S, s));
     if (io.feat_out) { Scope p(c, PC_EMBED, (double)M * D * 6, s); FREE_TRY(convert_rows(m.dtype, (long long)M * D, w.x, io.feat_out, s)); }
     FREE_TRY(run_head(c, w, st, S, w.head_out, s));
