@@ -15,9 +15,10 @@
 //              The whole warp runs the issue loop converged and one elected lane issues: measured on B200, a
 //              single-lane (divergent) loop of wait + 4 MMAs + commit takes ~660 clocks per K step, the converged
 //              loop ~508, and one MMA cannot be issued faster than every ~94 clocks whatever its size.  Only
-//              N = 256 (128 clocks of tensor work per instruction) therefore keeps the tensor core busy, so the
-//              tile is always 256 wide and a ragged last column block is zero-filled by TMA (rows of W past N)
-//              and clipped on the way out;
+//              N = 256 (128 clocks of tensor work per instruction) therefore keeps the tensor core busy, so tiles are
+//              256 wide; a ragged last column block (N = 1152 = 4.5 tiles) is computed only as wide as it is (its own
+//              tensor map of half as many W rows per CTA, its own instruction shape): it then runs at the
+//              shared-memory limit, 0.73 of a full tile's time instead of all of it;
 //   warps 2-5  epilogue (both CTAs, each on its own 128 rows): tcgen05.ld, fused bias / GELU / gate, then
 //              through swizzled shared-memory staging to a TMA store, or a TMA add-reduction for the gated
 //              residual update (the fp32 residual stream is never read by the SM).  QKV variants: HEADS scatters
@@ -46,6 +47,7 @@ constexpr uint32_t kSmemBudget = 227 * 1024;
 
 struct Tc2Args {
     int M, N, K, num_m, num_n, stages;
+    int last_n;                             // valid columns of the last column block (BN when N is a multiple of BN)
     const float* bias;
     const float* gate; long long gate_stride; int rows_per_seq;
     int heads, d_head, d_pad, n_tok;
@@ -94,7 +96,7 @@ __device__ __forceinline__ void scatter_qkv(const Tc2Args& a, int row, int n0, c
 template <int EPI, bool OUT_BF16, int BN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapW,
-                  const __grid_constant__ CUtensorMap mapO, const __grid_constant__ CUtensorMap mapV, const Tc2Args a) {
+                  const __grid_constant__ CUtensorMap mapWl, const __grid_constant__ CUtensorMap mapO, const __grid_constant__ CUtensorMap mapV, const Tc2Args a) {
     constexpr uint32_t kBBytes = (BN / 2) * BK * 2;          // one CTA's half of the W tile of a stage
     constexpr uint32_t kStageBytes = kABytes + kBBytes;
     extern __shared__ uint8_t smem_raw[];
@@ -132,22 +134,26 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
-        if (lane == 0) { tc::tma_prefetch_desc(&mapA); tc::tma_prefetch_desc(&mapW); }
+        if (lane == 0) { tc::tma_prefetch_desc(&mapA); tc::tma_prefetch_desc(&mapW); tc::tma_prefetch_desc(&mapWl); }
         const uint32_t full0 = tc::mapa(tc::smem_u32(&full[0]), 0);          // the even CTA's stage barriers
         int s = 0;                                           // stage and its phase advance by counting (no divisions in the loop)
         uint32_t ph = 0;
         bool ok = true;
         for (long long t = first; ok && t < total; t += step) {
             const int m_blk = (int)(t / a.num_n), n_blk = (int)(t % a.num_n);
-            const int a_row = m_blk * 256 + (int)rank * 128, w_row = n_blk * BN + (int)rank * (BN / 2);
+            // a ragged last column block is computed only as wide as it is: each CTA loads half of its valid W rows
+            const bool narrow = n_blk == a.num_n - 1 && a.last_n < BN;
+            const int half = narrow ? a.last_n / 2 : BN / 2;
+            const int a_row = m_blk * 256 + (int)rank * 128, w_row = n_blk * BN + (int)rank * half;
+            const uint32_t tx = 2u * (kABytes + (uint32_t)half * BK * 2u);
             for (int kb = 0; kb < nk; ++kb) {
                 ok = __all_sync(0xffffffffu, !*abort_flag && tc::mbar_wait(&empty[s], ph ^ 1u));
                 if (!ok) { if (lane == 0) fail(FREE_DEV_ERR_EMPTY_WAIT); break; }
                 if (tc::elect_one()) {
                     const uint32_t dst = tc::smem_u32(tiles + (size_t)s * kStageBytes);
-                    if (rank == 0) tc::mbar_expect_tx(&full[s], 2 * kStageBytes);
+                    if (rank == 0) tc::mbar_expect_tx(&full[s], tx);
                     tc::tma_load_2d_pair(dst, &mapA, full0 + 8u * s, kb * BK, a_row);
-                    tc::tma_load_2d_pair(dst + kABytes, &mapW, full0 + 8u * s, kb * BK, w_row);
+                    tc::tma_load_2d_pair(dst + kABytes, narrow ? &mapWl : &mapW, full0 + 8u * s, kb * BK, w_row);
                 }
                 __syncwarp();
                 if (++s == stages) { s = 0; ph ^= 1u; }
@@ -162,7 +168,7 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (even CTA only)
         if (rank == 0) {
-            const uint32_t idesc = tc::idesc_bf16(256, BN);
+            const uint32_t idesc_full = tc::idesc_bf16(256, BN), idesc_last = tc::idesc_bf16(256, a.last_n);
             uint32_t tl = 0, ph = 0;
             int s = 0;
             bool ok = true;
@@ -172,6 +178,7 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
                 if (!ok) { if (lane == 0) fail(FREE_DEV_ERR_ACC_EMPTY); break; }
                 tc::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * (uint32_t)BN;
+                const uint32_t idesc = (int)(t % a.num_n) == a.num_n - 1 ? idesc_last : idesc_full;
                 for (int kb = 0; kb < nk; ++kb) {
                     ok = __all_sync(0xffffffffu, !*abort_flag && tc::mbar_wait(&full[s], ph));
                     if (!ok) { if (lane == 0) fail(FREE_DEV_ERR_FULL_WAIT); break; }
@@ -366,8 +373,8 @@ int sm_count() {
 }
 
 template <int EPI, bool OUT_BF16, int BN>
-int launch(const CUtensorMap& mA, const CUtensorMap& mW, const CUtensorMap& mO, const CUtensorMap& mV, const Tc2Args& a, size_t smem,
-           cudaStream_t s) {
+int launch(const CUtensorMap& mA, const CUtensorMap& mW, const CUtensorMap& mWl, const CUtensorMap& mO, const CUtensorMap& mV,
+           const Tc2Args& a, size_t smem, cudaStream_t s) {
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] {
@@ -377,7 +384,7 @@ int launch(const CUtensorMap& mA, const CUtensorMap& mW, const CUtensorMap& mO, 
     const long long tiles = (long long)a.num_m * a.num_n;
     const long long pairs = sm_count() / 2;
     const int grid = 2 * (int)(tiles < pairs ? tiles : pairs);
-    linear_tc2_kernel<EPI, OUT_BF16, BN><<<grid, kThreads, smem, s>>>(mA, mW, mO, mV, a);
+    linear_tc2_kernel<EPI, OUT_BF16, BN><<<grid, kThreads, smem, s>>>(mA, mW, mWl, mO, mV, a);
     return free_check_launch();
 }
 
@@ -392,27 +399,30 @@ int dispatch(const LinearArgs& l, Tc2Args a, cudaStream_t s) {
     CUtensorMap mA, mW, mO;
     FREE_TRY(free_tensor_map_2d(&mA, l.A, (uint64_t)l.K, (uint64_t)l.M, (uint64_t)lda * 2, BK, 128, 128));
     FREE_TRY(free_tensor_map_2d(&mW, l.W, (uint64_t)l.K, (uint64_t)l.N, (uint64_t)ldw * 2, BK, BN / 2, 128));
+    a.last_n = l.N - (a.num_n - 1) * BN;                 // 64, 128, 192 or BN (N is a multiple of 64)
+    CUtensorMap mWl = mW;
+    if (a.last_n < BN) FREE_TRY(free_tensor_map_2d(&mWl, l.W, (uint64_t)l.K, (uint64_t)l.N, (uint64_t)ldw * 2, BK, (uint32_t)a.last_n / 2, 128));
     const bool ob = l.out_dtype == FREE_BF16;
     switch (l.epi) {
         case EPI_BIAS:
             FREE_TRY(free_tensor_map_2d_typed(&mO, ob ? 2 : 4, l.out, (uint64_t)l.N, (uint64_t)l.M, (uint64_t)ldo * (ob ? 2 : 4), ob ? 64 : 32, 32, 128));
-            return ob ? launch<EPI_BIAS, true, BN>(mA, mW, mO, mO, a, smem, s) : launch<EPI_BIAS, false, BN>(mA, mW, mO, mO, a, smem, s);
+            return ob ? launch<EPI_BIAS, true, BN>(mA, mW, mWl, mO, mO, a, smem, s) : launch<EPI_BIAS, false, BN>(mA, mW, mWl, mO, mO, a, smem, s);
         case EPI_BIAS_GELU:
             FREE_TRY(free_tensor_map_2d_typed(&mO, 2, l.out, (uint64_t)l.N, (uint64_t)l.M, (uint64_t)ldo * 2, 64, 32, 128));
-            return launch<EPI_BIAS_GELU, true, BN>(mA, mW, mO, mO, a, smem, s);
+            return launch<EPI_BIAS_GELU, true, BN>(mA, mW, mWl, mO, mO, a, smem, s);
         case EPI_GATE_RESIDUAL:
             FREE_TRY(free_tensor_map_2d_typed(&mO, 4, l.resid, (uint64_t)l.N, (uint64_t)l.M, (uint64_t)l.N * 4, 32, 32, 128));
-            return launch<EPI_GATE_RESIDUAL, false, BN>(mA, mW, mO, mO, a, smem, s);
+            return launch<EPI_GATE_RESIDUAL, false, BN>(mA, mW, mWl, mO, mO, a, smem, s);
         case EPI_QKV_HEADS:
             mO = mA;                                         // unused by this variant
-            return launch<EPI_QKV_HEADS, true, BN>(mA, mW, mO, mO, a, smem, s);
+            return launch<EPI_QKV_HEADS, true, BN>(mA, mW, mWl, mO, mO, a, smem, s);
         case EPI_QKV_TOKV: {
             CUtensorMap mV;
             const int qk_cols = 2 * l.heads * l.d_head;
             FREE_TRY(free_tensor_map_2d_typed(&mO, 2, l.out, (uint64_t)qk_cols, (uint64_t)l.M, (uint64_t)ldo * 2, 64, 32, 128));
             FREE_TRY(free_tensor_map_2d_typed(&mV, 2, l.vt, (uint64_t)l.n_tok, (uint64_t)(l.M / l.n_tok) * l.heads * l.d_pad,
                                               (uint64_t)l.n_tok * 2, 128, 8, 0));
-            return launch<EPI_QKV_TOKV, true, BN>(mA, mW, mO, mV, a, smem, s);
+            return launch<EPI_QKV_TOKV, true, BN>(mA, mW, mWl, mO, mV, a, smem, s);
         }
         default:
             return FREE_ERR_UNSUPPORTED;
