@@ -69,9 +69,9 @@ def test_dit_s2_guided_and_drafter(free):
         assert nerr(x_hat[i], mo_i + np.sqrt(sc.sigma2[t2[i]]) * z[i]) < TOL
 
 
-def test_bf16_trajectory_teacher_forced(free):
-    # the sampling loop in bf16 mode on a small model: every round's decisions must be the oracle verifier's
-    # decisions on the GPU's own means; checked through the final statistics of an all-accept and an all-reject run
+def test_bf16_trajectory_bounding_regimes(free):
+    # the sampling loop in bf16 mode on a small model, through the final statistics of an all-accept run, an
+    # (almost) all-reject run and the plain sampler; single rounds are checked draft by draft in the teacher-forced tests
     import dataclasses
     sh = dataclasses.replace(synth.DIT_S2, depth=2, H=16, W=16)
     N, K, B = 12, 3, 2
@@ -93,6 +93,18 @@ def test_bf16_trajectory_teacher_forced(free):
     # K = 0: plain sampler, N target calls per sample
     xf3, st3 = model.sample_trajectory(cu(x0), labels, dsched, 0, 0.0, cu(zt))
     assert st3["target_calls"] == B * N
+
+
+@pytest.mark.parametrize("cfg", [0.0, 3.0])
+def test_round_teacher_forced_small(free, cfg):
+    import dataclasses
+    from gpu_util import check_round_teacher_forced
+    sh = dataclasses.replace(synth.DIT_S2, depth=2, H=16, W=32)
+    w = synth.make_target_weights(sh, 5, bf16=True, ada_std=0.2, out_gain=2.0)
+    wd = synth.make_drafter_weights(sh, 6, bf16=True, ada_std=0.2, out_gain=2.0)
+    model = free.Model(sh, w, wd, dtype="bf16")
+    n = check_round_teacher_forced(free, model, sh, 50, np.array([3, 10, 20, 30, 41], np.int64), np.array([1, 2, 3, 4, 5], np.int32), 4, cfg, 21)
+    assert n.tolist() == [0, 1, 2, 3, 4]
 
 
 def test_ragged_row_blocks_and_single_query_tile(free):

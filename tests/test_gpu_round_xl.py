@@ -63,6 +63,15 @@ def test_xl_round_consistency(xl):
     assert torch.isfinite(x1).all() and torch.isfinite(x2).all()
 
 
+def test_xl_round_teacher_forced(xl):
+    # the benchmark's round (XL/2 512^2, guidance, K = 6) at batch 3: free_spec_round against the same round assembled
+    # from the public calls and against the oracle's verifier on the GPU's own means
+    from gpu_util import check_round_teacher_forced
+    free, sh, w, wd, model = xl
+    n = check_round_teacher_forced(free, model, sh, 250, np.array([5, 120, 240], np.int64), np.array([7, 400, 999], np.int32), 6, 4.0, 33)
+    assert n.tolist() == [0, 1, 2]
+
+
 def test_xl_256_packed_pass_sampled_against_oracle():
     # DiT-XL/2-shaped at 256^2: 256 tokens, B = 8 samples x K = 6 states, guidance scale 4 (96 sequences in one pass)
     import paper_2511_20390_b200 as free
