@@ -29,6 +29,7 @@ def parse():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--workload", default="default")
     ap.add_argument("--batch", type=int, default=0, help="images per step (0 = workload default)")
+    ap.add_argument("--graph", action="store_true", help="trajectory workload: replay the rounds as a CUDA graph")
     ap.add_argument("--res", type=int, default=512, choices=[256, 512], help="trajectory workload: image resolution")
     ap.add_argument("--chunk", type=int, default=0, help="verifier_fused: drafts per early-exit chunk (0 = off)")
     ap.add_argument("--no-cpu-baseline", action="store_true")

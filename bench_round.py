@@ -258,20 +258,24 @@ def run_trajectory(args):
     model.sample_trajectory(x0, labels, sched, K_DRAFTS, CFG, zt, zd, regimes["all_accepted"][1])      # warm-up
     torch.cuda.synchronize()
     out = {}
-    for name, (K, u) in regimes.items():
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        x, st = model.sample_trajectory(x0, labels, sched, K, CFG, zt, zd if K else None, u)
-        e1.record()
-        torch.cuda.synchronize()
-        sec = e0.elapsed_time(e1) / 1e3
-        assert torch.isfinite(x).all()
-        out[name] = {"images_per_s": B / sec, "seconds": sec, "rounds": st["rounds"], "target_calls": st["target_calls"],
-                     "draft_calls": st["draft_calls"], "accepted": st["accepted"], "rejected": st["rejected"],
-                     "parallel_efficiency": st["parallel_efficiency"]}
+    side = torch.cuda.Stream()            # the legacy default stream cannot be captured into a graph
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for name, (K, u) in regimes.items():
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            x, st = model.sample_trajectory(x0, labels, sched, K, CFG, zt, zd if K else None, u, use_graph=getattr(args, "graph", False))
+            e1.record()
+            torch.cuda.synchronize()
+            sec = e0.elapsed_time(e1) / 1e3
+            assert torch.isfinite(x).all()
+            out[name] = {"images_per_s": B / sec, "seconds": sec, "rounds": st["rounds"], "target_calls": st["target_calls"],
+                         "draft_calls": st["draft_calls"], "accepted": st["accepted"], "rejected": st["rejected"],
+                         "parallel_efficiency": st["parallel_efficiency"], "graph_rounds": st["graph_rounds"]}
     line = {"metric": "images/s", "value": out["all_accepted"]["images_per_s"], "unit": "images/s", "n_gpus": 1,
             "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": f"sample_trajectory, DiT-XL/2-shaped {res}^2, {N_SCHED} transitions, K={K_DRAFTS}, cfg {CFG}, batch {B}; "
+            "config": {"workload": f"sample_trajectory, DiT-XL/2-shaped {res}^2, {N_SCHED} transitions, K={K_DRAFTS}, cfg {CFG}, batch {B}"
+                                   f"{', rounds replayed as a CUDA graph' if getattr(args, 'graph', False) else ''}; "
                                    "value = the all-accepted regime"},
             "regimes": out}
     print(json.dumps(line))

@@ -223,6 +223,15 @@ typedef struct free_spec_params {
     int32_t K;                 /* drafts per round (0 = plain sequential sampler) */
     float   cfg_scale;
     const float* lambda;       /* DEVICE fp32 [N] relaxation table indexed by transition n-1 (n = 1 first), or NULL = strict */
+    int32_t use_graph;         /* sample_trajectory / free_uncertainty_profile only.  Non-zero: the second round is recorded
+                                  by stream capture into a CUDA graph and every later round is one graph launch (the rounds
+                                  of a trajectory launch the same kernels with the same arguments; what changes lives in the
+                                  workspace).  Removes the launch overhead that shows at small batches (4% per round at
+                                  B = 1 on XL/2 512^2).  The graph and its executable are driver objects created and
+                                  destroyed inside the call; `stream` must not be capturing already.  Ignored while
+                                  free_profile_begin() is active and on streams that cannot be captured (the legacy
+                                  default stream): the rounds are then launched one kernel at a time as usual.  free_spec_round() ignores the field: it can itself be
+                                  captured by the caller once it has run eagerly once. */
 } free_spec_params;
 
 typedef struct free_traj_stats {     /* HOST, filled on return */
@@ -232,6 +241,7 @@ typedef struct free_traj_stats {     /* HOST, filled on return */
     int64_t accepted, rejected;      /* drafts accepted / rejected, summed over samples */
     int64_t accept_hist[FREE_MAX_K + 1];   /* rounds that accepted exactly i drafts */
     double  parallel_efficiency;     /* B * N / target_calls (Sec. 4, metric 1) */
+    int64_t graph_rounds;            /* rounds launched as a CUDA graph (0 unless params->use_graph took effect) */
 } free_traj_stats;
 
 /*

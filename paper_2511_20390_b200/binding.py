@@ -46,7 +46,7 @@ class ScheduleDesc(C.Structure):
 
 
 class SpecParams(C.Structure):
-    _fields_ = [("K", C.c_int32), ("cfg_scale", C.c_float), ("lam", C.c_void_p)]
+    _fields_ = [("K", C.c_int32), ("cfg_scale", C.c_float), ("lam", C.c_void_p), ("use_graph", C.c_int32)]
 
 
 class ProfEntry(C.Structure):
@@ -56,7 +56,8 @@ class ProfEntry(C.Structure):
 class TrajStats(C.Structure):
     _fields_ = [("rounds", C.c_int64), ("target_calls", C.c_int64), ("draft_calls", C.c_int64),
                 ("accepted", C.c_int64), ("rejected", C.c_int64),
-                ("accept_hist", C.c_int64 * (FREE_MAX_K + 1)), ("parallel_efficiency", C.c_double)]
+                ("accept_hist", C.c_int64 * (FREE_MAX_K + 1)), ("parallel_efficiency", C.c_double),
+                ("graph_rounds", C.c_int64)]
 
 
 _LIB = None
@@ -469,11 +470,11 @@ class Model:
         return dev, acc, cnt
 
     def sample_trajectory(self, x0, labels, sched: DeviceSchedule, K, cfg_scale, noise_target, noise_draft=None,
-                          uniforms=None, lam=None):
+                          uniforms=None, lam=None, use_graph=False):
         """Algorithm 1 for a batch.  Returns (x_final, stats dict)."""
         B = x0.shape[0]
         _dev(x0, torch.float32); _dev(labels, torch.int32); _dev(noise_target, torch.float32)
-        prm = SpecParams(int(K), float(cfg_scale), None if lam is None else _dev(lam, torch.float32).data_ptr())
+        prm = SpecParams(int(K), float(cfg_scale), None if lam is None else _dev(lam, torch.float32).data_ptr(), int(bool(use_graph)))
         st = TrajStats()
         x_final = torch.empty_like(x0)
         ws = self.workspace(B * max(int(K), 1))
@@ -481,7 +482,7 @@ class Model:
                                        _ptr(noise_target), _ptr(noise_draft), _ptr(uniforms), _ptr(x_final),
                                        C.byref(st), _ptr(ws), ws.numel(), _stream()), "sample_trajectory")
         stats = {k: getattr(st, k) for k in ("rounds", "target_calls", "draft_calls", "accepted", "rejected",
-                                             "parallel_efficiency")}
+                                             "parallel_efficiency", "graph_rounds")}
         stats["accept_hist"] = list(st.accept_hist)[:int(K) + 1]
         return x_final, stats
 

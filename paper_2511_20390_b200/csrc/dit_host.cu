@@ -644,12 +644,42 @@ int run_trajectory(free_ctx* c, int B, const float* x0, const int32_t* labels, c
     }
     RoundIO r{B, K, labels, sch, prm->cfg_scale, prm->lambda, noise_target, noise_draft, uniforms};
 
+    // Every round launches the same kernels with the same arguments (cursors and states live in the workspace), so on
+    // request the second round is recorded into a CUDA graph and the later ones are single graph launches.
+    struct GraphHolder {
+        cudaGraphExec_t exec = nullptr;
+        ~GraphHolder() { if (exec) cudaGraphExecDestroy(exec); }
+    } gh;
+    bool want_graph = prm->use_graph && !c->prof_on;
     for (long long round = 0; round < 2LL * N + 2; ++round) {
         bool any = false;
         for (int b = 0; b < B; ++b) any |= h_a[b] <= N;
         if (!any) break;
         h_prev = h_a;
-        FREE_TRY(one_round(c, w, r, s));
+        if (!gh.exec && want_graph && round == 1) {          // round 0 ran eagerly: one-time function attributes are set
+            if (cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+                (void)cudaGetLastError();                  // e.g. the legacy default stream cannot be captured: stay eager
+                want_graph = false;
+            } else {
+                cudaGraph_t graph = nullptr;
+                const int rc = one_round(c, w, r, s);
+                const cudaError_t ce = cudaStreamEndCapture(s, &graph);
+                if (rc != FREE_OK || ce != cudaSuccess || !graph) {
+                    if (graph) cudaGraphDestroy(graph);
+                    (void)cudaGetLastError();
+                    return rc != FREE_OK ? rc : FREE_ERR_CUDA;
+                }
+                const cudaError_t ie = cudaGraphInstantiate(&gh.exec, graph, 0);
+                cudaGraphDestroy(graph);
+                if (ie != cudaSuccess) { gh.exec = nullptr; (void)cudaGetLastError(); return FREE_ERR_CUDA; }
+            }
+        }
+        if (gh.exec) {
+            FREE_CUDA_TRY(cudaGraphLaunch(gh.exec, s));
+            if (stats) stats->graph_rounds += 1;
+        } else {
+            FREE_TRY(one_round(c, w, r, s));
+        }
         FREE_CUDA_TRY(cudaMemcpyAsync(h_act.data(), w.active, B * 4, cudaMemcpyDeviceToHost, s));
         FREE_CUDA_TRY(cudaMemcpyAsync(h_nv.data(), w.nv, B * 4, cudaMemcpyDeviceToHost, s));
         if (K > 0) FREE_CUDA_TRY(cudaMemcpyAsync(h_acc.data(), w.n_acc, B * 4, cudaMemcpyDeviceToHost, s));

@@ -124,3 +124,44 @@ def test_ragged_row_blocks_and_single_query_tile(free):
     assert model.device_error() == 0
     mo, eo, fo = odit.verify_pass(w, sh, sc, x, t, y, 0.0)
     assert max(nerr(eps, eo), nerr(mean, mo), nerr(feat, fo)) < TOL
+
+
+def test_rounds_as_cuda_graphs(free):
+    """The rounds of a trajectory replayed as one CUDA graph (use_graph) and a round captured by the caller: both must
+    reproduce the eager launches bit for bit (same kernels, same arguments, state in the workspace)."""
+    import dataclasses
+    sh = dataclasses.replace(synth.DIT_S2, depth=2, H=16, W=32)
+    N, K, B, cfg = 20, 3, 3, 2.0
+    dsched = free.DeviceSchedule(free.respaced_schedule(N))
+    shape = (sh.C, sh.H, sh.W)
+    x0 = cu(synth.normal(4, 1, (B,) + shape))
+    zt, zd = cu(synth.normal(4, 2, (B, N) + shape)), cu(synth.normal(4, 3, (B, N) + shape))
+    u = cu(synth.uniform01(4, 4, (B, N)) * 1e-30)                    # a mix: tiny uniforms accept most drafts, not all
+    labels = cu(np.array([3, 7, 11], np.int32), torch.int32)
+    model = free.Model(sh, synth.make_target_weights(sh, 1, bf16=True), synth.make_drafter_weights(sh, 2, bf16=True), dtype="bf16")
+    x_e, st_e = model.sample_trajectory(x0, labels, dsched, K, cfg, zt, zd, u)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        x_g, st_g = model.sample_trajectory(x0, labels, dsched, K, cfg, zt, zd, u, use_graph=True)
+    torch.cuda.synchronize()
+    assert st_e["rounds"] >= 3 and st_e["graph_rounds"] == 0 and st_g["graph_rounds"] == st_g["rounds"] - 1
+    assert torch.equal(x_e, x_g) and {k: v for k, v in st_e.items() if k != "graph_rounds"} == {k: v for k, v in st_g.items() if k != "graph_rounds"}
+    # the legacy default stream cannot be captured: the request is ignored there
+    x_d, st_d = model.sample_trajectory(x0, labels, dsched, K, cfg, zt, zd, u, use_graph=True)
+    assert torch.equal(x_e, x_d) and st_d["graph_rounds"] in (0, st_d["rounds"] - 1)
+    # a round captured by the caller, after one eager call
+    cursor = cu(np.array([2, 9, 15], np.int32), torch.int32)
+    out = [torch.empty_like(x0), torch.empty_like(cursor), torch.zeros(B, dtype=torch.int32, device="cuda")]
+    ref = [t.clone() for t in model.spec_round(x0, cursor, labels, dsched, K, cfg, zt, zd, u)]
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            model.spec_round(x0, cursor, labels, dsched, K, cfg, zt, zd, u, x_next=out[0], cursor_next=out[1], n_accept=out[2])
+    torch.cuda.synchronize()
+    for _ in range(2):
+        for t in out:
+            t.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert all(torch.equal(a, b) for a, b in zip(out, ref)) and model.device_error() == 0
