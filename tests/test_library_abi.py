@@ -43,7 +43,8 @@ def test_struct_layouts_match_the_header(libpath):
     assert ctypes.sizeof(b.ModelDesc) == 12 * 4 + 8 * 8 + 80 + 4 * 8
     assert ctypes.sizeof(b.DrafterDesc) == 8 + 2 * 8 + 80 + 4 * 8
     assert ctypes.sizeof(b.ScheduleDesc) == 8 + 4 * 8
-    assert ctypes.sizeof(b.TrajStats) == 5 * 8 + 65 * 8 + 8
+    assert ctypes.sizeof(b.TrajStats) == 5 * 8 + 65 * 8 + 8 + 8
+    assert ctypes.sizeof(b.SpecParams) == 4 + 4 + 8 + 8            # K, cfg_scale, lambda, use_graph (+ padding)
 
 
 def test_argument_errors_need_no_gpu(libpath):
