@@ -88,6 +88,7 @@ CASES = [
     ((4, 64, 64), 2, 2, 33),         # K = 33
     ((4, 192, 192), 2, 1, 3),        # large latent
     ((4, 64, 64), 2, 200, 2),        # batch wide enough to narrow the clusters
+    ((4, 16, 16), 2, 2, 64),         # the largest K
 ]
 
 
@@ -169,6 +170,10 @@ def test_argument_errors():
         _run(dict(i, eps=np.concatenate([i["eps"], i["eps"][:, :, :1]], axis=2)), 4.0)
     L = free.lib()
     assert L.spec_verify_fused(1, 0, 16, 1, 1.0, *([None] * 10), 0, *([None] * 6)) != 0
+    t = cu(np.zeros(16, np.float32))
+    p = t.data_ptr()
+    assert L.spec_verify_fused(0, 2, 8, 1, 1.0, p, p, p, p, p, p, p, None, p, None, 0, p, p, None, None, None, None) == 0      # empty batch
+    assert L.spec_verify_fused(1, 65, 8, 1, 1.0, p, p, p, p, p, p, p, None, p, None, 0, p, p, None, None, None, None) == -2    # K too large
 
 
 def test_full_size_point_sampled_against_oracle():
