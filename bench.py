@@ -284,10 +284,14 @@ class DrafterLossWorkload:
         torch.cuda.current_stream().synchronize()
         return sum(t.numel() * t.element_size() for t in self.pinned), 32
 
+    # DRAM bytes (read + write) of one launch at 64 samples from the ncu capture summarised in
+    # profiles/loss_partial_kernel_xl512_64samples.txt; traffic is proportional to the batch
+    NCU_DRAM_BYTES_64 = 313.7e6
+
     def roofline(self, ms_per_step, peaks):
         ach = self.bytes_per_step / 1e9 / (ms_per_step / 1e3)
         return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
-                "traffic": None, "kernel": "loss_partial_kernel", "peak_source": peaks["source"]}
+                "traffic": self.NCU_DRAM_BYTES_64 * self.n / 64.0, "kernel": "loss_partial_kernel", "peak_source": peaks["source"]}
 
     def oracle_sample(self):
         from oracle import losses as ol
