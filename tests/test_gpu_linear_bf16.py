@@ -19,7 +19,8 @@ def _operands(M, N, K, seed):
 
 SHAPES = [(128, 32, 64), (128, 256, 64), (256, 192, 128), (300, 384, 192), (96, 64, 256), (1, 128, 64),
           (1000, 1152, 1152), (777, 3456, 384), (40000, 384, 64), (19500, 160, 128), (640, 4608, 1152), (512, 1152, 4608),
-          (9000, 3456, 384), (6100, 4608, 128), (129, 192, 64), (300, 320, 128), (2049, 1152, 256)]
+          (9000, 3456, 384), (6100, 4608, 128), (129, 192, 64), (300, 320, 128), (2049, 1152, 256),
+          (700, 448, 128), (515, 704, 192), (260, 256, 64)]        # last column block 192, 192 and none: every narrow width of the CTA-pair kernel
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES)
