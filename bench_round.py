@@ -22,6 +22,15 @@ def round_flops(shape, B, K, G, n_draft_blocks=1):
     return B * G * seq + K * B * G * draft + B * K * G * seq
 
 
+def round_config(B, K, G):
+    """The `config` object of the round workload (shared by the CUDA arm and the oracle arm of the benchmark)."""
+    return {"workload": f"FREE round, DiT-XL/2-shaped 512^2 (latent 4x64x64, 1024 tokens, width 1152, 28 blocks, "
+                        f"16 heads), K={K} drafts, cfg {CFG} (doubled batch), batch {B}, 1-block drafter, "
+                        f"{N_SCHED}-step schedule",
+            "B": B, "K": K, "sequences_in_packed_pass": B * K * G,
+            "cache": "activations per step (several GB) exceed L2"}
+
+
 class RoundWorkload:
     metric = "DiT-XL/2 512^2 packed-verify TFLOP/s"
     unit = "TFLOP/s"
@@ -53,11 +62,7 @@ class RoundWorkload:
         self.G = 2
         self.flops = round_flops(sh, B, K, self.G)
         self.units_per_step = self.flops / 1e12
-        self.config = {"workload": f"FREE round, DiT-XL/2-shaped 512^2 (latent 4x64x64, 1024 tokens, width 1152, 28 blocks, "
-                                   f"16 heads), K={K} drafts, cfg {CFG} (doubled batch), batch {B}, 1-block drafter, "
-                                   f"{N_SCHED}-step schedule",
-                       "B": B, "K": K, "sequences_in_packed_pass": B * K * self.G,
-                       "cache": "activations per step (several GB) exceed L2"}
+        self.config = round_config(B, K, self.G)
         # host staging for the end-to-end path
         pin = lambda t: torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t)
         self.h_in = [pin(self.x_cur), pin(self.cursor), pin(self.labels)]
@@ -171,7 +176,7 @@ def reference_arm(args, cores):
     dt = (time.perf_counter() - t0) / max(args.steps, 1)
     val = float(np.mean(vals))
     return {"metric": RoundWorkload.metric, "value": val, "unit": "TFLOP/s", "ms_per_step": dt * 1e3, "dtype": "f64",
-            "config": {"workload": "FREE round, DiT-XL/2-shaped 512^2, K=6, cfg 4, batch 16 (oracle: bounded sample)"},
+            "config": round_config(args.batch or 16, K_DRAFTS, 2),
             "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample}}
 
 
