@@ -1,0 +1,43 @@
+"""The benchmark's JSON lines on reduced batches: every workload runs through the public API and reports the keys the
+measurement contract names (a guard for bench.py itself; the numbers are not judged here)."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+
+pytestmark = pytest.mark.gpu
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _line(*args):
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), *args], capture_output=True, text=True, timeout=600, cwd=ROOT)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    return json.loads(lines[0])
+
+
+@pytest.mark.parametrize("args,bound", [
+    (("--batch", "1", "--steps", "2", "--no-cpu-baseline"), "tensor"),
+    (("--workload", "verifier", "--batch", "16", "--steps", "3", "--no-cpu-baseline"), "hbm"),
+    (("--workload", "verifier_fused", "--batch", "16", "--steps", "3", "--chunk", "4"), "hbm"),
+    (("--workload", "drafter_loss", "--batch", "8", "--steps", "3", "--no-cpu-baseline"), "hbm"),
+])
+def test_bench_line(args, bound):
+    d = _line(*args)
+    for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling", "vs_baseline",
+                "dtype", "data", "config", "clocks", "e2e", "gpu_launches", "roofline"):
+        assert key in d, key
+    assert d["n_gpus"] == 1 and d["warmup"] >= 3 and d["value"] > 0 and d["ms_per_step"] > 0 and d["gpu_launches"] > 0
+    assert d["data"] == "synthetic" and "workload" in d["config"] and "model" not in d["config"]
+    rf = d["roofline"]
+    assert rf["bound"] == bound and rf["achieved"] > 0 and rf["peak"] > 0 and abs(rf["frac"] - rf["achieved"] / rf["peak"]) < 1e-9
+    assert "traffic" in rf and rf["unit"] in ("GB/s", "TFLOP/s")
+    e = d["e2e"]
+    assert e["value"] > 0 and e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] > 0 and e["unit"] == d["unit"]
+    assert {"sm_mhz", "sm_max_mhz", "reasons"} <= set(d["clocks"])
+    if "--no-cpu-baseline" not in args:
+        c = d["cpu_baseline"]
+        assert c["kind"] == "oracle" and c["value"] > 0 and c["cores"] >= 1 and c["sample"]
