@@ -213,3 +213,26 @@ def test_trajectory_with_other_variance_schedules(free, kw):
         assert nerr(xf[b], xo) < 5 * TOL
         acc += so["accepted"]; rej += so["rejected"]
     assert st["accepted"] == acc and st["rejected"] == rej and acc + rej > 10
+
+
+def test_trajectory_with_more_drafts_than_transitions(free):
+    """K larger than the whole schedule: every round drafts up to the last but one transition (the final, noise-free
+    transition is never drafted) and the loop still matches the oracle."""
+    sh, w, wd, model = _tiny_model(free)
+    N, B, K, cfg = 6, 2, 9, 0.0
+    sc = osched.make("linear", N)
+    dsched = free.DeviceSchedule(free.linear_schedule(N))
+    shape = (sh.C, sh.H, sh.W)
+    x0 = synth.normal(24, 1, (B,) + shape)
+    zt, zd = synth.normal(24, 2, (B, N) + shape), synth.normal(24, 3, (B, N) + shape)
+    u = synth.uniform01(24, 4, (B, N)) * 1e-3                       # small uniforms: most drafts are accepted
+    labels = np.array([0, 9], np.int32)
+    xf, st = model.sample_trajectory(cu(x0), cu(labels, torch.int32), dsched, K, cfg, cu(zt), cu(zd), cu(u))
+    acc = rej = calls = 0
+    for b in range(B):
+        xo, so, trace = _oracle_traj(sh, w, wd, sc, N, K, cfg, x0[b], int(labels[b]), zt[b], zd[b], u[b])
+        assert all(abs(ell - np.log(u[b, t - 1])) > 1e-3 for t, ok, ell in trace if ell < 0)
+        assert max(t for t, _, _ in trace) <= N - 1                 # the last transition is never verified as a draft
+        assert nerr(xf[b], xo) < 5 * TOL
+        acc += so["accepted"]; rej += so["rejected"]; calls += so["target_calls"]
+    assert st["accepted"] == acc and st["rejected"] == rej and st["target_calls"] == calls
