@@ -84,6 +84,91 @@ __global__ void __launch_bounds__(256) patch_embed_kernel(int n_items, int G, in
     }
 }
 
+// Wide models (D a multiple of 128, 16-value patches): the transposed weight matrix [16][D] sits in shared memory, a warp
+// takes four consecutive tokens at a time and a lane the same 4-column groups of all of them, so that every 16-byte
+// weight read feeds 16 multiply-adds and every store is a full row segment.  Bound by the output's HBM bandwidth.
+template <typename T, int VPL>
+__global__ void __launch_bounds__(256, 2) patch_embed_wide_kernel(int n_items, int G, int C, int H, int W, int p, int D,
+                                                                  const float* __restrict__ x_in, long long x_stride,
+                                                                  const float* __restrict__ pe_w, const float* __restrict__ pe_b,
+                                                                  const float* __restrict__ pos, T* __restrict__ out) {
+    constexpr int PD = 16, TOKW = 4;
+    extern __shared__ float4 pe_smem[];
+    float* wt = reinterpret_cast<float*>(pe_smem);                    // [PD][D]
+    float* patches = wt + (size_t)PD * D;                             // [warps][TOKW][PD]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpc = blockDim.x >> 5;
+    for (int i = threadIdx.x; i < PD * D; i += blockDim.x) { const int o = i / PD, e = i % PD; wt[(size_t)e * D + o] = pe_w[i]; }
+    __syncthreads();
+    float* mine = patches + warp * TOKW * PD;
+    const int gw = W / p, n_tok = (H / p) * gw;
+    const int n_groups = n_items / TOKW;                              // the host checks n_tok % TOKW == 0
+    const int warps = gridDim.x * wpc;
+    auto gather2 = [&](int group, float& a, float& b) {               // this lane's two of the group's 64 patch values
+        const int e = lane & 15;
+        const int c = e / (p * p), r = (e / p) % p, cc = e % p;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int item = group * TOKW + (lane >> 4) + 2 * h;
+            const int st = item / n_tok, tok = item % n_tok, ti = tok / gw, tj = tok % gw;
+            const float v = x_in[(long long)st * x_stride + ((long long)c * H + ti * p + r) * W + tj * p + cc];
+            if (h == 0) a = v; else b = v;
+        }
+    };
+    int group = blockIdx.x * wpc + warp;
+    float na = 0.f, nb = 0.f;
+    if (group < n_groups) gather2(group, na, nb);
+    for (; group < n_groups; group += warps) {
+        __syncwarp();
+        mine[(lane >> 4) * PD + (lane & 15)] = na;
+        mine[((lane >> 4) + 2) * PD + (lane & 15)] = nb;
+        __syncwarp();
+        if (group + warps < n_groups) gather2(group + warps, na, nb);  // the next group's values while this one is computed
+        float pt[TOKW][PD];
+#pragma unroll
+        for (int t = 0; t < TOKW; ++t)
+#pragma unroll
+            for (int e4 = 0; e4 < PD / 4; ++e4) {
+                const float4 v = reinterpret_cast<const float4*>(mine + t * PD)[e4];
+                pt[t][4 * e4] = v.x; pt[t][4 * e4 + 1] = v.y; pt[t][4 * e4 + 2] = v.z; pt[t][4 * e4 + 3] = v.w;
+            }
+        const int item0 = group * TOKW, st = item0 / n_tok, tok0 = item0 % n_tok;   // four tokens of one state
+#pragma unroll 1
+        for (int i = 0; i < VPL; ++i) {
+            const int c0 = (i * 32 + lane) * 4;
+            const float4 bias = __ldg(reinterpret_cast<const float4*>(pe_b + c0));
+            float4 acc[TOKW];
+#pragma unroll
+            for (int t = 0; t < TOKW; ++t) {
+                const float4 ps = __ldg(reinterpret_cast<const float4*>(pos + (long long)(tok0 + t) * D + c0));
+                acc[t] = make_float4(bias.x + ps.x, bias.y + ps.y, bias.z + ps.z, bias.w + ps.w);
+            }
+#pragma unroll
+            for (int e = 0; e < PD; ++e) {
+                const float4 w4 = *reinterpret_cast<const float4*>(wt + (size_t)e * D + c0);
+#pragma unroll
+                for (int t = 0; t < TOKW; ++t) {
+                    acc[t].x = fmaf(w4.x, pt[t][e], acc[t].x); acc[t].y = fmaf(w4.y, pt[t][e], acc[t].y);
+                    acc[t].z = fmaf(w4.z, pt[t][e], acc[t].z); acc[t].w = fmaf(w4.w, pt[t][e], acc[t].w);
+                }
+            }
+#pragma unroll
+            for (int t = 0; t < TOKW; ++t)
+                for (int g = 0; g < G; ++g) {
+                    T* dst = out + ((long long)(st * G + g) * n_tok + tok0 + t) * D + c0;
+                    if (sizeof(T) == 4) {
+                        *reinterpret_cast<float4*>(dst) = acc[t];
+                    } else {
+                        __nv_bfloat162 lo = __floats2bfloat162_rn(acc[t].x, acc[t].y), hi = __floats2bfloat162_rn(acc[t].z, acc[t].w);
+                        uint2 pk;
+                        pk.x = *reinterpret_cast<uint32_t*>(&lo);
+                        pk.y = *reinterpret_cast<uint32_t*>(&hi);
+                        *reinterpret_cast<uint2*>(dst) = pk;
+                    }
+                }
+        }
+    }
+}
+
 // Any patch size / width: one CTA per (state, token), weights read from global memory.
 template <typename T>
 __global__ void __launch_bounds__(128) patch_embed_generic_kernel(int G, int C, int H, int W, int p, int D,
@@ -316,6 +401,24 @@ static int patch_embed_launch(int n_states, int G, int C, int H, int W, int p, i
                               const float* pe_w, const float* pe_b, const float* pos, T* out, cudaStream_t s) {
     const int n_tok = (H / p) * (W / p), pd = C * p * p;
     const int n_items = n_states * n_tok;
+    if (pd == 16 && D % 128 == 0 && D / 128 <= 9 && n_tok % 4 == 0 && free_aligned16(pe_b) && free_aligned16(pos) && free_aligned16(out)) {
+        const int vpl = D / 128, wpc = 8;
+        const size_t smem = (size_t)16 * D * 4 + (size_t)wpc * 4 * 16 * 4;
+        const int n_groups = n_items / 4;
+        const unsigned need = (unsigned)((n_groups + wpc - 1) / wpc), cap = 148u * 2u;
+        const unsigned grid = need < cap ? need : cap;
+        cudaError_t attr = cudaSuccess;
+#define FREE_PE_WIDE(V) do { static cudaError_t once = cudaFuncSetAttribute(patch_embed_wide_kernel<T, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * 128 * V * 4 + 8 * 4 * 16 * 4); attr = once; \
+            if (attr == cudaSuccess) patch_embed_wide_kernel<T, V><<<grid, 256, smem, s>>>(n_items, G, C, H, W, p, D, x_in, x_stride, pe_w, pe_b, pos, out); } while (0)
+        switch (vpl) {
+            case 3: FREE_PE_WIDE(3); break;
+            case 9: FREE_PE_WIDE(9); break;
+            default: attr = cudaErrorInvalidValue; break;
+        }
+#undef FREE_PE_WIDE
+        if (attr == cudaSuccess) return free_check_launch();
+        (void)cudaGetLastError();                         // other widths: the kernels below
+    }
     if (pd == 16 && D <= 5 * 256) {                   // the DiT */2 models: 4 channels, 2 x 2 patches
         const unsigned grid = (unsigned)(n_items < 148 * 4 ? n_items : 148 * 4);
         const int cpt = (D + 255) / 256;
