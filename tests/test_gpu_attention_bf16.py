@@ -37,3 +37,33 @@ def test_attention_peaked_rows():
     got = b.op_attention(cu(qkv.reshape(1, T, 3 * dh), torch.bfloat16), h)
     ref = odit.attention(*(qkv[0, :, i, 0].astype(np.float64) for i in range(3)))
     assert nerr(got[0], ref) < 1e-2
+
+
+@pytest.mark.parametrize("T,h,dh", [(1024, 2, 72), (512, 1, 64), (384, 1, 96)])
+def test_attention_offset_moves_in_every_block(T, h, dh):
+    # logits along one direction grow from one block of 128 keys to the next by far more than the threshold at which
+    # the exponent offset of a row is moved: rows with a positive projection rescale their accumulator in every block,
+    # rows with a negative one keep the offset of their first block while later keys underflow to zero
+    from paper_2511_20390_b200 import binding as b
+    rng = np.random.default_rng(T + dh)
+    e = rng.standard_normal(dh)
+    e /= np.linalg.norm(e)
+    sign = np.where(rng.random((T, 1)) < 0.5, -1.0, 1.0)
+    qkv = np.zeros((1, T, 3, h, dh), np.float32)
+    for a in range(h):
+        q = sign * 3.0 * np.sqrt(dh) ** 0.5 * e + 0.3 * rng.standard_normal((T, dh))
+        step = (np.arange(T) // 128 + 1.0)[:, None]                 # 1, 2, ... per block of keys
+        k = step * 4.0 * np.sqrt(dh) ** 0.5 * e + 0.3 * rng.standard_normal((T, dh))
+        qkv[0, :, 0, a], qkv[0, :, 1, a], qkv[0, :, 2, a] = q, k, rng.standard_normal((T, dh))
+    qkv = synth.round_to_bf16(qkv)
+    got = b.op_attention(cu(qkv.reshape(1, T, 3 * h * dh), torch.bfloat16), h)
+    torch.cuda.synchronize()
+    for a in range(h):
+        q64, k64, v64 = (qkv[0, :, i, a].astype(np.float64) for i in range(3))
+        logits = q64 @ k64.T / np.sqrt(dh)
+        rising = logits[:, -128:].max(1) - logits[:, :128].max(1)
+        thr = 8.0 * (T // 128 - 1)                                  # ~11 per block of keys
+        assert (rising > thr).sum() > T // 4 and (rising < -thr).sum() > T // 4   # both kinds of row are present
+        ref = odit.attention(q64, k64, v64)
+        assert np.isfinite(got[0, :, a * dh:(a + 1) * dh].float().cpu().numpy()).all()
+        assert nerr(got[0, :, a * dh:(a + 1) * dh], ref) < 1e-2, a
