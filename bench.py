@@ -461,7 +461,7 @@ def main():
                "gpu_launches": int(round(wl.launches_per_step * args.steps)),
                "roofline": wl.roofline(kernel_ms, peaks)}
         if hasattr(wl, "extra"):
-            out.update(wl.extra(ms_step, peaks))
+            out.update(wl.extra(ms_step, dict(peaks, sm_mhz=clocks["sm_mhz"] if clocks else None)))
         if world == 1 and not args.no_cpu_baseline:
             v, sample = wl.oracle_sample()
             out["cpu_baseline"] = {"value": v, "unit": wl.unit, "cores": cpu_threads(), "kind": "oracle", "sample": sample}

@@ -139,7 +139,17 @@ class RoundWorkload:
                 e["gbs"] = round(p["work"] / 1e9 / (p["ms"] / 1e3), 1)
             kern.append(e)
         value = self.flops / 1e12 / (ms_step / 1e3)
-        return {"pct_of_bf16_peak": {"of_measured_sustained": value / peaks["bf16_tflops_sustained"],
+        more = {}
+        att = next((e for e in kern if e["name"] == "attention" and "tflops" in e), None)
+        if att and peaks.get("sm_mhz"):
+            # attention at d_head 72 is bounded by the exp2 unit, not the tensor core: 16 exponentials per clock per SM,
+            # one per score, and a score stands for 4 d_head algorithmic FLOPs (its share of Q K^T and of P V)
+            n_sm = self.torch.cuda.get_device_properties(0).multi_processor_count
+            peak = 16.0 * n_sm * peaks["sm_mhz"] * 1e6 * 4.0 * self.shape.d_head / 1e12
+            more["attention_roofline"] = {"bound": "alu", "achieved": att["tflops"], "peak": round(peak, 1), "unit": "TFLOP/s",
+                                          "frac": round(att["tflops"] / peak, 4), "kernel": "attention_tc2_kernel",
+                                          "peak_source": "exp2 unit: 16 per clock per SM x SMs x median SM clock of this run x 4 d_head FLOP"}
+        return {**more, "pct_of_bf16_peak": {"of_measured_sustained": value / peaks["bf16_tflops_sustained"],
                                      "of_measured_burst": value / peaks["bf16_tflops"], "of_nominal_2250": value / 2250.0},
                 "images_per_s_if_all_accepted": self.B * (K_DRAFTS + 1) / N_SCHED / (ms_step / 1e3),
                 "kernels": kern}

@@ -35,6 +35,9 @@ def test_bench_line(args, bound):
     rf = d["roofline"]
     assert rf["bound"] == bound and rf["achieved"] > 0 and rf["peak"] > 0 and abs(rf["frac"] - rf["achieved"] / rf["peak"]) < 1e-9
     assert "traffic" in rf and rf["unit"] in ("GB/s", "TFLOP/s")
+    if bound == "tensor":
+        ar = d["attention_roofline"]                            # the round also reports its exp2-bound kernel
+        assert ar["bound"] == "alu" and ar["peak"] > 0 and 0 < ar["frac"] < 1.5
     e = d["e2e"]
     assert e["value"] > 0 and e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] > 0 and e["unit"] == d["unit"]
     assert {"sm_mhz", "sm_max_mhz", "reasons"} <= set(d["clocks"])
