@@ -70,7 +70,7 @@ __device__ __forceinline__ float ex2(float x) { float y; asm("ex2.approx.ftz.f32
 template <int DP>
 __global__ void __launch_bounds__(kThreads, 1)
 attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_constant__ CUtensorMap mapQK1,
-                     const __grid_constant__ CUtensorMap mapV, const Attn2Args a) {
+                     const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapO, const Attn2Args a) {
     using G = Geo2<DP>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -131,7 +131,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
         const int row_q = seq * T + q0;                     // row of the first query in the token-major matrix
         const int xq = a.q_col0 + head * a.d_head, xk = a.k_col0 + head * a.d_head;
         const int v_row = sh * DP;
-        if (lane == 0) { tc::tma_prefetch_desc(&mapQK0); tc::tma_prefetch_desc(&mapV); }
+        if (lane == 0) { tc::tma_prefetch_desc(&mapQK0); tc::tma_prefetch_desc(&mapV); tc::tma_prefetch_desc(&mapO); }
         if (tc::elect_one()) {
             tc::mbar_expect_tx(bar_q, (uint32_t)nq * G::QK_BYTES);
             for (int t = 0; t < nq; ++t) {
@@ -361,11 +361,17 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
             l_x[(t * 2 + hf) * 128 + r] = l_run;
             pair_sync();
             if (ok) ok = wait(&o_full[t], (uint32_t)(nb - 1) & 1u);
+            // The rows leave through shared memory: every thread puts its normalised columns into a dense row-major copy
+            // of the tile (in the tile's P buffer, which the last P V has finished reading), and one TMA store per 32 rows
+            // writes whole row segments.  (Per-thread 16-byte stores to 32 different rows per instruction kept the
+            // load/store unit busy for some 3000 clocks per CTA with nothing else left to overlap them.)
+            const uint32_t row_bytes = (uint32_t)a.d_head * 2u;
+            uint8_t* stage = tiles + G::OFF_P + t * G::P_BYTES;
             if (ok) {
                 tc::tc_fence_after();
                 const float inv = 1.f / (l_run + l_x[(t * 2 + (hf ^ 1)) * 128 + r]);
-                __nv_bfloat16* dst = a.out + ((long long)seq * T + q0 + t * BQ + r) * ((long long)a.heads * a.d_head) + (long long)head * a.d_head;
                 const int dh = a.d_head;                            // multiple of 8
+                uint8_t* srow = stage + (uint32_t)r * row_bytes;
                 for (int ch = ch0; ch < ch1; ++ch) {
                     const int c0 = ch * 16;
                     uint32_t ov[16];
@@ -380,9 +386,18 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
                                 __nv_bfloat162 bb = __floats2bfloat162_rn(__uint_as_float(ov[h8 + 2 * i]) * inv, __uint_as_float(ov[h8 + 2 * i + 1]) * inv);
                                 w[i] = *reinterpret_cast<uint32_t*>(&bb);
                             }
-                            *reinterpret_cast<uint4*>(dst + c0 + h8) = make_uint4(w[0], w[1], w[2], w[3]);
+                            *reinterpret_cast<uint4*>(srow + (c0 + h8) * 2) = make_uint4(w[0], w[1], w[2], w[3]);
                         }
                     }
+                }
+                tc::fence_proxy_async();                            // the staged rows are read by the TMA unit
+            }
+            pair_sync();                                            // both column halves of these 32 rows are in place
+            if (ok) {
+                if (hf == 0 && lane == 0) {
+                    tc::tma_store_2d(&mapO, tc::smem_u32(stage + (uint32_t)(wq * 32) * row_bytes), head * a.d_head, seq * T + q0 + t * BQ + wq * 32);
+                    tc::bulk_commit();
+                    tc::bulk_wait_read<0>();                        // shared memory is given back when the CTA ends
                 }
             } else if (lane == 0) {
                 fail();
@@ -406,14 +421,16 @@ int launch(int n_seq, int n_tok, int heads, int d_head, const void* qk, long lon
     if (attr_err != cudaSuccess) return FREE_ERR_CUDA;
     const uint64_t rows = (uint64_t)n_seq * n_tok, rows_v = (uint64_t)n_seq * heads * DP;
     if (rows > 0x7fffffffull || rows_v > 0x7fffffffull) return FREE_ERR_SHAPE;
-    CUtensorMap mQK0, mQK1, mV;
+    CUtensorMap mQK0, mQK1, mV, mO;
     FREE_TRY(free_tensor_map_2d(&mQK0, qk, (uint64_t)width, rows, (uint64_t)ld * 2, 64, 128, 128));
     if (G::W1 > 0) FREE_TRY(free_tensor_map_2d(&mQK1, qk, (uint64_t)width, rows, (uint64_t)ld * 2, G::W1, 128, (int)G::ROW1));
     else mQK1 = mQK0;
     FREE_TRY(free_tensor_map_2d(&mV, vt, (uint64_t)n_tok, rows_v, (uint64_t)n_tok * 2, 64, DP, 128));
+    // output rows [n_seq * n_tok, heads * d_head]: boxes of one head's columns x 32 rows, dense in shared memory
+    FREE_TRY(free_tensor_map_2d(&mO, out, (uint64_t)heads * d_head, rows, (uint64_t)heads * d_head * 2, (uint32_t)d_head, 32, 0));
     Attn2Args a{n_tok, heads, d_head, q_col0, k_col0, 1.4426950408889634f / sqrtf((float)d_head), (__nv_bfloat16*)out, err};
     dim3 grid((n_tok + 2 * BQ - 1) / (2 * BQ), n_seq * heads);
-    attention_tc2_kernel<DP><<<grid, kThreads, G::SMEM, s>>>(mQK0, mQK1, mV, a);
+    attention_tc2_kernel<DP><<<grid, kThreads, G::SMEM, s>>>(mQK0, mQK1, mV, mO, a);
     return free_check_launch();
 }
 
