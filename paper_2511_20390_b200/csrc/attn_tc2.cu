@@ -1,12 +1,21 @@
 // Non-causal multi-head self-attention on the 5th-generation tensor cores, two query tiles per CTA.
 //
-// One CTA (one per SM) owns 256 queries of one (sequence, head): two tiles of 128 queries that alternate on the
-// tensor core, so that the softmax of one tile runs while the MMAs of the other execute.
+// A work item is 256 queries of one (sequence, head): two tiles of 128 queries that alternate on the tensor core and on
+// the exp2 unit, so that the softmax of one tile runs while the MMAs of the other execute.  CTAs are persistent (one
+// per SM) and walk over the items: at d_head 72 and 1024 tokens an item is only 8 key blocks long, and launching,
+// allocating TMEM, loading Q and filling the pipeline once per item cost a quarter of the time.  The producer loads the
+// next item's Q (as soon as the last S of the current item has read the old one), K and V, and the next item's first S
+// is issued, while the softmax warps still finish, normalise and store the current item.
+// Phases.  The exp2 phases of the two tiles must alternate: when they coincide each takes 2200 clocks instead of 1350
+// and nothing overlaps the rest of a block (4000 clocks per block instead of 3300).  Nothing restores the alternation
+// once it is lost, and the end of an item leaves the tiles skewed, so every item starts with a hand-over: tile 1 takes
+// its first block after tile 0's first, and tile 0 its second block after tile 1's first.
 //   warps 0-7   softmax of query tile 0: a query row (= one TMEM lane) is shared by two threads, warp w and warp
 //               w + 4, which take the two halves of 64 keys of every block (four softmax warps per scheduler keep
 //               the exp2 unit, which bounds this kernel at d_head 72, fed while others wait on TMEM or barriers)
 //   warps 8-15  the same for query tile 1
-//   warp 16     TMA producer: Q tiles once, then K and V^T blocks of 128 keys into double buffers
+//   warp 16     TMA producer: per item the Q tiles (whose padding columns it zeroes itself), then K and V^T blocks of
+//               128 keys into double buffers
 //   warps 17-18 MMA issuers, one per query tile (each runs converged, one elected lane issues; a barrier poll costs
 //               ~200 clocks and an MMA issue ~50-100, so one warp serving both tiles was the bottleneck):
 //               S_t = Q_t K^T (128 x 128 x d_pad) into TMEM, O_t = P_t V (128 x d_pad x 128) into TMEM
@@ -17,7 +26,9 @@
 // warps) so that both use the same exponent offset, and add their partial row sums at the end.  O_t accumulates in TMEM across all key blocks: the exponent offset of a row is only moved when the row
 // maximum has grown by more than 8 (a factor 256), in which case the row's O and running sum are rescaled in place
 // before that block's P V is issued; numerator and denominator always share the offset, so the result is exact.
-// Issue order per block: S_0(next), PV_0, S_1(next), PV_1.
+// Issue order per block and tile: S(next), then P V; at an item's last block P V first (the next S waits for the next
+// item's operands).  The finished rows are normalised into a dense copy of the tile in shared memory (the tile's P
+// buffer) and leave by one TMA store per 32 rows.
 //
 // Operands.  q and k are read straight from a token-major bf16 matrix [n_seq * n_tok, ld] (the output of the QKV
 // linear layer): head h of q starts at column q_col0 + h * d_head, of k at k_col0 + h * d_head.  d_pad is 64 plus a
@@ -38,9 +49,9 @@ constexpr uint32_t kTmemCols = 512;           // S_0 [0,128), S_1 [128,256), O_0
 
 struct Attn2Args {
     int n_tok, heads, d_head;
+    int n_items, qblocks;                    // work items = (sequence * heads + head, block of 256 queries)
     int q_col0, k_col0;
     float scale_log2e;
-    __nv_bfloat16* out;
     uint32_t* err;
 };
 
@@ -84,24 +95,29 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
     uint64_t* p_ready = bar_q + 12;     // [2] per tile: P stored and S consumed (4 warp arrivals)
     uint64_t* o_full = bar_q + 14;      // [2] per tile: O_j complete
     uint64_t* s_free = bar_q + 16;      // [2] per tile: S_j read out of TMEM (4 warp arrivals)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_q + 18);
+    uint64_t* q_free = bar_q + 18;      // the last S of an item has read Q (one commit per tile): the next item's Q may land
+    uint64_t* o_free = bar_q + 19;      // [2] per tile: the finished O has been read out of TMEM (8 warp arrivals)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_q + 21);
     volatile uint32_t* abort_flag = tmem_slot + 1;
     float* mx_x = reinterpret_cast<float*>(smem + 1024);       // [parity][tile][half][row]
     float* l_x = reinterpret_cast<float*>(smem + 5120);        // [tile][half][row]
     uint8_t* tiles = smem + kCtrlBytes;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int sh = blockIdx.y;                              // sequence * heads + head
-    const int seq = sh / a.heads, head = sh % a.heads;
-    const int q0 = blockIdx.x * 2 * BQ;
     const int T = a.n_tok, nb = T / BKV;
-    const int nq = (q0 + BQ < T) ? 2 : 1;                   // query tiles this CTA really has
+    // The CTA walks over work items first, first + step, ...  All its items have the same number of query tiles: the
+    // host launches one CTA per item when the last block of 256 queries is half empty.
+    const int first = blockIdx.x, step = gridDim.x;
+    const int nq = ((first % a.qblocks) * 2 * BQ + BQ < T) ? 2 : 1;
+    const int my_items = first < a.n_items ? (a.n_items - first + step - 1) / step : 0;
+    const uint32_t total = (uint32_t)my_items * (uint32_t)nb;          // key blocks this CTA goes through
 
     if (threadIdx.x == 0) {
-        tc::mbar_init(bar_q, 1); tc::mbar_init(bar_qz, 4 * nq);
+        tc::mbar_init(bar_q, 1); tc::mbar_init(bar_qz, 1); tc::mbar_init(q_free, nq);
         for (int i = 0; i < 2; ++i) {
             tc::mbar_init(&k_full[i], 1); tc::mbar_init(&k_empty[i], nq); tc::mbar_init(&v_full[i], 1); tc::mbar_init(&v_empty[i], nq);
             tc::mbar_init(&s_full[i], 1); tc::mbar_init(&p_ready[i], 8); tc::mbar_init(&o_full[i], 1); tc::mbar_init(&s_free[i], 8);
+            tc::mbar_init(&o_free[i], 8);
         }
         *abort_flag = 0;
         tc::fence_barrier_init();
@@ -127,42 +143,73 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
     };
 
     if (warp == 16) {
-        // ------------------------------------------------------------------ TMA producer
-        const int row_q = seq * T + q0;                     // row of the first query in the token-major matrix
-        const int xq = a.q_col0 + head * a.d_head, xk = a.k_col0 + head * a.d_head;
-        const int v_row = sh * DP;
-        if (lane == 0) { tc::tma_prefetch_desc(&mapQK0); tc::tma_prefetch_desc(&mapV); tc::tma_prefetch_desc(&mapO); }
-        if (tc::elect_one()) {
-            tc::mbar_expect_tx(bar_q, (uint32_t)nq * G::QK_BYTES);
-            for (int t = 0; t < nq; ++t) {
-                uint8_t* sQ = tiles + G::OFF_Q + t * G::QK_BYTES;
-                tc::tma_load_2d(sQ, &mapQK0, bar_q, xq, row_q + t * BQ);
-                if (G::W1 > 0) tc::tma_load_2d(sQ + G::QK0_BYTES, &mapQK1, bar_q, xq + 64, row_q + t * BQ);
-            }
-        }
-        __syncwarp();
+        // ------------------------------------------------------------------ TMA producer (and Q fix-up)
+        if (lane == 0) { tc::tma_prefetch_desc(&mapQK0); tc::tma_prefetch_desc(&mapV); }
         bool ok = true;
-        for (int j = 0; ok && j < nb; ++j) {
-            const int b = j & 1;
-            const uint32_t ph = (uint32_t)(j >> 1) & 1u;
-            ok = wait(&k_empty[b], ph ^ 1u);
-            if (!ok) break;
+        uint32_t g = 0;                                     // running key-block count: buffer g & 1, phase (g >> 1) & 1
+        int it = 0;
+        for (int w = first; ok && w < a.n_items; w += step, ++it) {
+            const int sh = w / a.qblocks, q0 = (w % a.qblocks) * 2 * BQ;       // sh = sequence * heads + head
+            const int seq = sh / a.heads, head = sh % a.heads;
+            const int row_q = seq * T + q0;                 // row of the first query in the token-major matrix
+            const int xq = a.q_col0 + head * a.d_head, xk = a.k_col0 + head * a.d_head;
+            const int v_row = sh * DP;
+            if (it > 0) {                                   // the previous item's last S has read the Q tiles
+                ok = wait(q_free, (uint32_t)(it - 1) & 1u);
+                if (!ok) break;
+            }
             if (tc::elect_one()) {
-                uint8_t* sK = tiles + G::OFF_K + b * G::QK_BYTES;
-                tc::mbar_expect_tx(&k_full[b], G::QK_BYTES);
-                tc::tma_load_2d(sK, &mapQK0, &k_full[b], xk, seq * T + j * BKV);
-                if (G::W1 > 0) tc::tma_load_2d(sK + G::QK0_BYTES, &mapQK1, &k_full[b], xk + 64, seq * T + j * BKV);
+                tc::mbar_expect_tx(bar_q, (uint32_t)nq * G::QK_BYTES);
+                for (int t = 0; t < nq; ++t) {
+                    uint8_t* sQ = tiles + G::OFF_Q + t * G::QK_BYTES;
+                    tc::tma_load_2d(sQ, &mapQK0, bar_q, xq, row_q + t * BQ);
+                    if (G::W1 > 0) tc::tma_load_2d(sQ + G::QK0_BYTES, &mapQK1, bar_q, xq + 64, row_q + t * BQ);
+                }
             }
             __syncwarp();
-            ok = wait(&v_empty[b], ph ^ 1u);
-            if (!ok) break;
-            if (tc::elect_one()) {
-                uint8_t* sV = tiles + G::OFF_V + b * G::V_BYTES;
-                tc::mbar_expect_tx(&v_full[b], G::V_BYTES);
-                tc::tma_load_2d(sV, &mapV, &v_full[b], j * BKV, v_row);
-                tc::tma_load_2d(sV + G::V_HALF, &mapV, &v_full[b], j * BKV + 64, v_row);
+            for (int j = 0; ok && j < nb; ++j, ++g) {
+                const int b = (int)(g & 1u);
+                const uint32_t ph = (g >> 1) & 1u;
+                ok = wait(&k_empty[b], ph ^ 1u);
+                if (!ok) break;
+                if (tc::elect_one()) {
+                    uint8_t* sK = tiles + G::OFF_K + b * G::QK_BYTES;
+                    tc::mbar_expect_tx(&k_full[b], G::QK_BYTES);
+                    tc::tma_load_2d(sK, &mapQK0, &k_full[b], xk, seq * T + j * BKV);
+                    if (G::W1 > 0) tc::tma_load_2d(sK + G::QK0_BYTES, &mapQK1, &k_full[b], xk + 64, seq * T + j * BKV);
+                }
+                __syncwarp();
+                if (j == 0) {
+                    // Q has landed: zero its columns [d_head, d_pad) (they belong to the next head), then release it to
+                    // the MMA warps.  Done here so that the next item's first S can be issued while the softmax warps
+                    // still finish the previous item.
+                    ok = wait(bar_q, (uint32_t)it & 1u);
+                    if (!ok) break;
+                    if constexpr (G::W1 > 0) {
+                        constexpr int units = G::ROW1 / 16, rows_per_128 = 128 / G::ROW1;
+                        for (int t = 0; t < nq; ++t) {
+                            uint8_t* sQ = tiles + G::OFF_Q + t * G::QK_BYTES;
+                            for (int r = lane; r < BQ; r += 32)
+                                for (int u = (a.d_head - 64) / 8; u < units; ++u) {
+                                    const int su = u ^ ((r / rows_per_128) & (units - 1));
+                                    *reinterpret_cast<uint4*>(sQ + G::QK0_BYTES + r * G::ROW1 + su * 16) = make_uint4(0u, 0u, 0u, 0u);
+                                }
+                        }
+                    }
+                    tc::fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(bar_qz);
+                }
+                ok = wait(&v_empty[b], ph ^ 1u);
+                if (!ok) break;
+                if (tc::elect_one()) {
+                    uint8_t* sV = tiles + G::OFF_V + b * G::V_BYTES;
+                    tc::mbar_expect_tx(&v_full[b], G::V_BYTES);
+                    tc::tma_load_2d(sV, &mapV, &v_full[b], j * BKV, v_row);
+                    tc::tma_load_2d(sV + G::V_HALF, &mapV, &v_full[b], j * BKV + 64, v_row);
+                }
+                __syncwarp();
             }
-            __syncwarp();
         }
         if (!ok) {
             if (lane == 0) fail();
@@ -200,11 +247,12 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
                 vd[0][k] = tc::smem_desc(v_base + half * G::V_HALF + ko, 1024, 2);
                 vd[1][k] = tc::smem_desc(v_base + G::V_BYTES + half * G::V_HALF + ko, 1024, 2);
             }
-            auto issue_s = [&](int kb) {                        // S_t = Q_t K^T over d_pad in steps of 16 (elected lane)
+            auto issue_s = [&](int kb, bool last_of_item) {     // S_t = Q_t K^T over d_pad in steps of 16 (elected lane)
 #pragma unroll
                 for (int k = 0; k < KS; ++k) tc::mma_bf16(d_s, qd[k], kb ? kd[1][k] : kd[0][k], idesc_s, k != 0);
                 tc::mma_commit(&s_full[t]);
                 tc::mma_commit(&k_empty[kb]);                   // one arrival per tile
+                if (last_of_item) tc::mma_commit(q_free);       // Q is no longer needed once this S has executed
             };
             auto issue_o = [&](int vb, uint32_t accumulate) {   // O_t (+)= P_t V over the 128 keys in steps of 16
 #pragma unroll
@@ -212,28 +260,51 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
                 tc::mma_commit(&o_full[t]);
                 tc::mma_commit(&v_empty[vb]);
             };
-            bool ok = wait2(bar_q, 0, bar_qz, 0) && wait(&k_full[0], 0);
+            bool ok = total > 0 && wait2(bar_q, 0, bar_qz, 0) && wait(&k_full[0], 0);
             if (ok) {
                 tc::tc_fence_after();
-                if (tc::elect_one()) issue_s(0);
+                if (tc::elect_one()) issue_s(0, nb == 1);
                 __syncwarp();
             }
-            for (int j = 0; ok && j < nb; ++j) {
-                const int b = j & 1;
-                const uint32_t ph = (uint32_t)j & 1u, bph = (uint32_t)(j >> 1) & 1u;
-                if (j + 1 < nb) {
-                    // S_t of the next block as soon as this tile's softmax has pulled S_t of this block out of TMEM
-                    ok = wait2(&s_free[t], ph, &k_full[b ^ 1], (uint32_t)((j + 1) >> 1) & 1u);
-                    if (!ok) break;
-                    tc::tc_fence_after();
-                    if (tc::elect_one()) issue_s(b ^ 1);
-                    __syncwarp();
+            int j = 0, it = 0;                                  // block within the item, item count
+            for (uint32_t g = 0; ok && g < total; ++g) {
+                const int b = (int)(g & 1u);
+                const uint32_t ph = g & 1u, bph = (g >> 1) & 1u;
+                const bool new_item = j + 1 == nb;
+                // Order within a block: the next block's S first (its operands are there long before this block's P).  At
+                // an item's last block the other way round: the next S needs the next item's Q and K, and this item's
+                // last P V must not wait for them.
+#pragma unroll 1
+                for (int stepi = 0; ok && stepi < 2; ++stepi) {
+                    const bool do_s = (stepi == 0) != new_item;
+                    if (do_s) {
+                        if (g + 1 < total) {
+                            // S_t of the next block (of this item or of the next one) as soon as this tile's softmax has
+                            // pulled S_t of this block out of TMEM
+                            ok = wait2(&s_free[t], ph, &k_full[b ^ 1], ((g + 1) >> 1) & 1u);
+                            if (!ok) break;
+                            if (new_item) {
+                                ok = wait2(bar_q, (uint32_t)(it + 1) & 1u, bar_qz, (uint32_t)(it + 1) & 1u);
+                                if (!ok) break;
+                            }
+                            tc::tc_fence_after();
+                            if (tc::elect_one()) issue_s(b ^ 1, new_item ? nb == 1 : j + 2 == nb);
+                            __syncwarp();
+                        }
+                    } else {
+                        ok = wait2(&p_ready[t], ph, &v_full[b], bph);
+                        if (!ok) break;
+                        if (j == 0 && it > 0) {                 // the previous item's O has been read out
+                            ok = wait(&o_free[t], (uint32_t)(it - 1) & 1u);
+                            if (!ok) break;
+                        }
+                        tc::tc_fence_after();
+                        if (tc::elect_one()) issue_o(b, j > 0 ? 1u : 0u);
+                        __syncwarp();
+                    }
                 }
-                ok = wait2(&p_ready[t], ph, &v_full[b], bph);
                 if (!ok) break;
-                tc::tc_fence_after();
-                if (tc::elect_one()) issue_o(b, j > 0 ? 1u : 0u);
-                __syncwarp();
+                if (++j == nb) { j = 0; ++it; }
             }
             if (!ok && lane == 0) fail();
         }
@@ -245,27 +316,10 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
             const int r = wq * 32 + lane;                          // query row within the tile = TMEM lane
             const uint32_t lane_sel = (uint32_t)(wq * 32) << 16;
             const uint32_t tmem_S = tmem_base + t * 128 + hf * 64 + lane_sel, tmem_O = tmem_base + 256 + t * 128 + lane_sel;
-            uint8_t* sQ = tiles + G::OFF_Q + t * G::QK_BYTES;
             uint8_t* prow = tiles + G::OFF_P + t * G::P_BYTES + hf * G::P_HALF + r * 128;   // this thread's 64 keys of P
             constexpr int NCH = DP / 16;                            // 16-column chunks of O: the two threads of a row split them
             const int ch0 = hf == 0 ? 0 : (NCH + 1) / 2, ch1 = hf == 0 ? (NCH + 1) / 2 : NCH;
             bool ok = true;
-            if (hf == 0) {
-                ok = wait(bar_q, 0);
-                if (ok) {
-                    // zero the Q columns [d_head, d_pad) of this row (they belong to the next head)
-                    if constexpr (G::W1 > 0) {
-                        constexpr int units = G::ROW1 / 16, rows_per_128 = 128 / G::ROW1;
-                        for (int u = (a.d_head - 64) / 8; u < units; ++u) {
-                            const int su = u ^ ((r / rows_per_128) & (units - 1));
-                            *reinterpret_cast<uint4*>(sQ + G::QK0_BYTES + r * G::ROW1 + su * 16) = make_uint4(0u, 0u, 0u, 0u);
-                        }
-                    }
-                    tc::fence_proxy_async();
-                    __syncwarp();
-                    if (lane == 0) tc::mbar_arrive(bar_qz);
-                }
-            }
             float m_used = -INFINITY, l_run = 0.f;                  // exponent offset of this row; sum over this thread's keys
             const float cs = a.scale_log2e;
             const int pair_id = 1 + t * 4 + wq;                     // named barrier of the two warps that share these rows
@@ -273,12 +327,14 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
             // The pair barrier is a hardware barrier (cheap, but unbounded): both warps therefore run it in every
             // iteration whatever happened before, and a warp whose bounded wait gave up only stops doing work.
             bool s_polled = false;                                  // an early poll already saw this block's S complete
-            for (int j = 0; j < nb; ++j) {
-                const uint32_t ph = (uint32_t)j & 1u;
+            int j = 0, w = first;                                   // block within the item, the item
+            for (uint32_t g = 0; g < total; ++g) {
+                const uint32_t ph = g & 1u;
                 uint32_t sv[64];                                    // this thread's half row of S
                 float m_half = 0.f;
                 bool o_polled = false;
-                float* xs = mx_x + (((j & 1) * 2 + t) * 2) * 128;
+                float* xs = mx_x + (((int)(g & 1u) * 2 + t) * 2) * 128;
+                if (j == 0) { m_used = -INFINITY; l_run = 0.f; }
                 if (ok && !s_polled) ok = wait(&s_full[t], ph);
                 if (ok) {
                     tc::tc_fence_after();
@@ -288,7 +344,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
                     __syncwarp();
                     if (lane == 0) tc::mbar_arrive(&s_free[t]);     // the next block's S may overwrite TMEM now
                     // poll early for the previous P V (its latency hides behind the maximum and the pair barrier)
-                    if (j > 0) o_polled = tc::mbar_try_wait(&o_full[t], ph ^ 1u);
+                    if (g > 0) o_polled = tc::mbar_try_wait(&o_full[t], ph ^ 1u);
                     float m0 = __uint_as_float(sv[0]), m1 = __uint_as_float(sv[1]), m2 = __uint_as_float(sv[2]), m3 = __uint_as_float(sv[3]);
 #pragma unroll
                     for (int i = 4; i < 64; i += 4) {
@@ -300,6 +356,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
                 }
                 pair_sync();
                 // the previous P V has read P and O_t is complete up to the previous block: P may be overwritten, O rescaled
+                // (within an item; at an item's first block the previous P V was awaited before O was read out)
                 if (ok && j > 0 && !__all_sync(0xffffffffu, o_polled)) ok = wait(&o_full[t], ph ^ 1u);
                 if (ok) {
                     const float m_new = fmaxf(m_used, fmaxf(m_half, xs[(hf ^ 1) * 128 + r]));
@@ -322,10 +379,13 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
                         }
                         m_used = m_new;
                     }
-                    // once, on the first block: tile 1 starts its exponentials when tile 0 has finished its own, so that
-                    // from then on one tile is in its exp2 phase (the unit both tiles share) while the other loads,
-                    // exchanges and stores
-                    if (j == 0 && t == 1) ok = wait(&p_ready[0], 0);
+                    // on the first block of every item: tile 1 starts its exponentials when tile 0 has finished its own,
+                    // so that from then on one tile is in its exp2 phase (the unit both tiles share) while the other
+                    // loads, exchanges and stores
+                    if (j == 0 && t == 1) ok = wait(&p_ready[0], ph);
+                    // and tile 0 takes its second block after tile 1's first: whatever skew the previous item left
+                    // between the tiles, they leave the item's start in opposite phases
+                    if (j == 1 && t == 0 && nq == 2) ok = wait(&p_ready[1], ph ^ 1u);
                 }
                 if (ok) {
                     const float mc = m_used * cs;
@@ -356,52 +416,57 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
                     if (lane == 0) tc::mbar_arrive(&p_ready[t]);
                     s_polled = __all_sync(0xffffffffu, s_next);
                 }
-            }
-            // row sum = this thread's keys + the partner's (both were kept at the same exponent offset)
-            l_x[(t * 2 + hf) * 128 + r] = l_run;
-            pair_sync();
-            if (ok) ok = wait(&o_full[t], (uint32_t)(nb - 1) & 1u);
-            // The rows leave through shared memory: every thread puts its normalised columns into a dense row-major copy
-            // of the tile (in the tile's P buffer, which the last P V has finished reading), and one TMA store per 32 rows
-            // writes whole row segments.  (Per-thread 16-byte stores to 32 different rows per instruction kept the
-            // load/store unit busy for some 3000 clocks per CTA with nothing else left to overlap them.)
-            const uint32_t row_bytes = (uint32_t)a.d_head * 2u;
-            uint8_t* stage = tiles + G::OFF_P + t * G::P_BYTES;
-            if (ok) {
-                tc::tc_fence_after();
-                const float inv = 1.f / (l_run + l_x[(t * 2 + (hf ^ 1)) * 128 + r]);
-                const int dh = a.d_head;                            // multiple of 8
-                uint8_t* srow = stage + (uint32_t)r * row_bytes;
-                for (int ch = ch0; ch < ch1; ++ch) {
-                    const int c0 = ch * 16;
-                    uint32_t ov[16];
-                    tc::tmem_ld16(tmem_O + c0, ov);
-                    tc::tmem_wait_ld();
+                if (++j < nb) continue;
+                // ---- the item's last block is done: normalise and store its rows, then hand O back
+                j = 0;
+                // row sum = this thread's keys + the partner's (both were kept at the same exponent offset)
+                l_x[(t * 2 + hf) * 128 + r] = l_run;
+                pair_sync();
+                if (ok) ok = wait(&o_full[t], ph);
+                const uint32_t row_bytes = (uint32_t)a.d_head * 2u;
+                uint8_t* stage = tiles + G::OFF_P + t * G::P_BYTES;
+                if (ok) {
+                    tc::tc_fence_after();
+                    const float inv = 1.f / (l_run + l_x[(t * 2 + (hf ^ 1)) * 128 + r]);
+                    const int dh = a.d_head;                            // multiple of 8
+                    uint8_t* srow = stage + (uint32_t)r * row_bytes;
+                    for (int ch = ch0; ch < ch1; ++ch) {
+                        const int c0 = ch * 16;
+                        uint32_t ov[16];
+                        tc::tmem_ld16(tmem_O + c0, ov);
+                        tc::tmem_wait_ld();
 #pragma unroll
-                    for (int h8 = 0; h8 < 16; h8 += 8) {
-                        if (c0 + h8 < dh) {
-                            uint32_t w[4];
+                        for (int h8 = 0; h8 < 16; h8 += 8) {
+                            if (c0 + h8 < dh) {
+                                uint32_t wv[4];
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                __nv_bfloat162 bb = __floats2bfloat162_rn(__uint_as_float(ov[h8 + 2 * i]) * inv, __uint_as_float(ov[h8 + 2 * i + 1]) * inv);
-                                w[i] = *reinterpret_cast<uint32_t*>(&bb);
+                                for (int i = 0; i < 4; ++i) {
+                                    __nv_bfloat162 bb = __floats2bfloat162_rn(__uint_as_float(ov[h8 + 2 * i]) * inv, __uint_as_float(ov[h8 + 2 * i + 1]) * inv);
+                                    wv[i] = *reinterpret_cast<uint32_t*>(&bb);
+                                }
+                                *reinterpret_cast<uint4*>(srow + (c0 + h8) * 2) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
                             }
-                            *reinterpret_cast<uint4*>(srow + (c0 + h8) * 2) = make_uint4(w[0], w[1], w[2], w[3]);
                         }
                     }
+                    tc::tc_fence_before();
+                    tc::fence_proxy_async();                            // the staged rows are read by the TMA unit
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(&o_free[t]);         // the next item's first P V may overwrite O
                 }
-                tc::fence_proxy_async();                            // the staged rows are read by the TMA unit
-            }
-            pair_sync();                                            // both column halves of these 32 rows are in place
-            if (ok) {
-                if (hf == 0 && lane == 0) {
+                pair_sync();                                            // both column halves of these 32 rows are in place
+                if (ok && hf == 0 && lane == 0) {
+                    const int sh = w / a.qblocks, q0 = (w % a.qblocks) * 2 * BQ;
+                    const int seq = sh / a.heads, head = sh % a.heads;
                     tc::tma_store_2d(&mapO, tc::smem_u32(stage + (uint32_t)(wq * 32) * row_bytes), head * a.d_head, seq * T + q0 + t * BQ + wq * 32);
                     tc::bulk_commit();
-                    tc::bulk_wait_read<0>();                        // shared memory is given back when the CTA ends
+                    tc::bulk_wait_read<0>();
                 }
-            } else if (lane == 0) {
-                fail();
+                // the staged rows share the tile's P buffer: every store of the tile has read its rows before any warp
+                // writes the next item's P (hardware barrier of the tile's 8 warps, run unconditionally like pair_sync)
+                asm volatile("bar.sync %0, 256;" ::"r"(9 + t) : "memory");
+                w += step;
             }
+            if (!ok && lane == 0) fail();
         }
     }
     tc::tc_fence_before();
@@ -426,10 +491,16 @@ int launch(int n_seq, int n_tok, int heads, int d_head, const void* qk, long lon
     if (G::W1 > 0) FREE_TRY(free_tensor_map_2d(&mQK1, qk, (uint64_t)width, rows, (uint64_t)ld * 2, G::W1, 128, (int)G::ROW1));
     else mQK1 = mQK0;
     FREE_TRY(free_tensor_map_2d(&mV, vt, (uint64_t)n_tok, rows_v, (uint64_t)n_tok * 2, 64, DP, 128));
-    // output rows [n_seq * n_tok, heads * d_head]: boxes of one head's columns x 32 rows, dense in shared memory
     FREE_TRY(free_tensor_map_2d(&mO, out, (uint64_t)heads * d_head, rows, (uint64_t)heads * d_head * 2, (uint32_t)d_head, 32, 0));
-    Attn2Args a{n_tok, heads, d_head, q_col0, k_col0, 1.4426950408889634f / sqrtf((float)d_head), (__nv_bfloat16*)out, err};
-    dim3 grid((n_tok + 2 * BQ - 1) / (2 * BQ), n_seq * heads);
+    const int qblocks = (n_tok + 2 * BQ - 1) / (2 * BQ);
+    const long long n_items = (long long)qblocks * n_seq * heads;
+    if (n_items > 0x7fffffffll) return FREE_ERR_SHAPE;
+    Attn2Args a{n_tok, heads, d_head, (int)n_items, qblocks, q_col0, k_col0, 1.4426950408889634f / sqrtf((float)d_head), err};
+    // persistent CTAs, one per SM, when every item has two query tiles; else one CTA per item (they then differ)
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { (void)cudaGetLastError(); sms = 148; }
+    const bool uniform = n_tok % (2 * BQ) == 0;
+    const unsigned grid = (unsigned)((uniform && n_items > sms) ? sms : n_items);
     attention_tc2_kernel<DP><<<grid, kThreads, G::SMEM, s>>>(mQK0, mQK1, mV, mO, a);
     return free_check_launch();
 }
@@ -448,17 +519,6 @@ int attention_tc2(int n_seq, int n_tok, int heads, int d_head, const void* qk, l
     if (!attention_tc2_supported(n_tok, d_head)) return FREE_ERR_UNSUPPORTED;
     if (ld % 8 || q_col0 % 8 || k_col0 % 8 || width > ld || !free_aligned16(qk) || !free_aligned16(vt) || !free_aligned16(out)) return FREE_ERR_ALIGN;
     const int dp = attention_tc2_dpad(d_head);
-    if ((long long)n_seq * heads > 65535) {
-        // grid.y limit: split the batch of sequences
-        const int per = 65535 / heads;
-        for (int s0 = 0; s0 < n_seq; s0 += per) {
-            const int ns = n_seq - s0 < per ? n_seq - s0 : per;
-            FREE_TRY(attention_tc2(ns, n_tok, heads, d_head, (const char*)qk + (size_t)s0 * n_tok * ld * 2, ld, width, q_col0, k_col0,
-                                   (const char*)vt + (size_t)s0 * heads * dp * n_tok * 2,
-                                   (char*)out + (size_t)s0 * n_tok * heads * d_head * 2, err, s));
-        }
-        return FREE_OK;
-    }
     switch (dp) {
         case 64: return launch<64>(n_seq, n_tok, heads, d_head, qk, ld, width, q_col0, k_col0, vt, out, err, s);
         case 80: return launch<80>(n_seq, n_tok, heads, d_head, qk, ld, width, q_col0, k_col0, vt, out, err, s);
