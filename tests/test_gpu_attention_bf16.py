@@ -12,7 +12,9 @@ pytestmark = pytest.mark.gpu
 
 @pytest.mark.parametrize("n_seq,T,h,dh,gain", [(2, 256, 6, 64, 1.0), (1, 1024, 2, 72, 1.0), (3, 128, 1, 64, 1.0),
                                                (1, 256, 2, 96, 1.0), (1, 256, 1, 128, 1.0), (1, 384, 2, 40, 1.0),
-                                               (2, 1024, 3, 72, 3.0), (5, 256, 16, 72, 0.3)])
+                                               (2, 1024, 3, 72, 3.0), (5, 256, 16, 72, 0.3),
+                                               # more work items than SMs: persistent CTAs take several items each
+                                               (10, 512, 16, 72, 1.0), (40, 256, 8, 64, 2.0), (3, 1024, 16, 72, 1.0)])
 def test_attention_tc(n_seq, T, h, dh, gain):
     from paper_2511_20390_b200 import binding as b
     qkv = synth.round_to_bf16(synth.normal(T + dh, 1, (n_seq, T, 3, h, dh), std=gain))
@@ -39,8 +41,8 @@ def test_attention_peaked_rows():
     assert nerr(got[0], ref) < 1e-2
 
 
-@pytest.mark.parametrize("T,h,dh", [(1024, 2, 72), (512, 1, 64), (384, 1, 96)])
-def test_attention_offset_moves_in_every_block(T, h, dh):
+@pytest.mark.parametrize("T,h,dh,n_seq", [(1024, 2, 72, 1), (512, 1, 64, 1), (384, 1, 96, 1), (1024, 2, 72, 20)])
+def test_attention_offset_moves_in_every_block(T, h, dh, n_seq):
     # logits along one direction grow from one block of 128 keys to the next by far more than the threshold at which
     # the exponent offset of a row is moved: rows with a positive projection rescale their accumulator in every block,
     # rows with a negative one keep the offset of their first block while later keys underflow to zero
@@ -56,8 +58,12 @@ def test_attention_offset_moves_in_every_block(T, h, dh):
         k = step * 4.0 * np.sqrt(dh) ** 0.5 * e + 0.3 * rng.standard_normal((T, dh))
         qkv[0, :, 0, a], qkv[0, :, 1, a], qkv[0, :, 2, a] = q, k, rng.standard_normal((T, dh))
     qkv = synth.round_to_bf16(qkv)
-    got = b.op_attention(cu(qkv.reshape(1, T, 3 * h * dh), torch.bfloat16), h)
+    # n_seq > 1: the same sequence many times, so that persistent CTAs go through several work items each; the copies
+    # must come out identical
+    got = b.op_attention(cu(np.repeat(qkv, n_seq, axis=0).reshape(n_seq, T, 3 * h * dh), torch.bfloat16), h)
     torch.cuda.synchronize()
+    for s_i in range(1, n_seq):
+        assert torch.equal(got[s_i], got[0]), s_i
     for a in range(h):
         q64, k64, v64 = (qkv[0, :, i, a].astype(np.float64) for i in range(3))
         logits = q64 @ k64.T / np.sqrt(dh)
