@@ -355,6 +355,13 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
                     xs[hf * 128 + r] = m_half;                      // for the thread that holds the other 64 keys of this row
                 }
                 pair_sync();
+                if (j == 0 && w != first) {
+                    // The previous item's rows were staged in the tile's P buffer: every store of the tile has read its
+                    // rows before any warp writes this item's P (the stores had the whole first part of this block to
+                    // do so; hardware barrier of the tile's 8 warps, run unconditionally like pair_sync).
+                    if (hf == 0 && lane == 0) tc::bulk_wait_read<0>();
+                    asm volatile("bar.sync %0, 256;" ::"r"(9 + t) : "memory");
+                }
                 // the previous P V has read P and O_t is complete up to the previous block: P may be overwritten, O rescaled
                 // (within an item; at an item's first block the previous P V was awaited before O was read out)
                 if (ok && j > 0 && !__all_sync(0xffffffffu, o_polled)) ok = wait(&o_full[t], ph ^ 1u);
@@ -458,14 +465,11 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
                     const int sh = w / a.qblocks, q0 = (w % a.qblocks) * 2 * BQ;
                     const int seq = sh / a.heads, head = sh % a.heads;
                     tc::tma_store_2d(&mapO, tc::smem_u32(stage + (uint32_t)(wq * 32) * row_bytes), head * a.d_head, seq * T + q0 + t * BQ + wq * 32);
-                    tc::bulk_commit();
-                    tc::bulk_wait_read<0>();
+                    tc::bulk_commit();                                  // read back before the next item's first P store
                 }
-                // the staged rows share the tile's P buffer: every store of the tile has read its rows before any warp
-                // writes the next item's P (hardware barrier of the tile's 8 warps, run unconditionally like pair_sync)
-                asm volatile("bar.sync %0, 256;" ::"r"(9 + t) : "memory");
                 w += step;
             }
+            if (hf == 0 && lane == 0) tc::bulk_wait_read<0>();          // shared memory is given back when the CTA ends
             if (!ok && lane == 0) fail();
         }
     }
