@@ -247,23 +247,24 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
                 vd[0][k] = tc::smem_desc(v_base + half * G::V_HALF + ko, 1024, 2);
                 vd[1][k] = tc::smem_desc(v_base + G::V_BYTES + half * G::V_HALF + ko, 1024, 2);
             }
-            auto issue_s = [&](int kb, bool last_of_item) {     // S_t = Q_t K^T over d_pad in steps of 16 (elected lane)
+            // The whole warp runs the issue sequences; the instructions are predicated on the elected lane `el`.
+            auto issue_s = [&](uint32_t el, int kb, bool last_of_item) {   // S_t = Q_t K^T over d_pad in steps of 16
 #pragma unroll
-                for (int k = 0; k < KS; ++k) tc::mma_bf16(d_s, qd[k], kb ? kd[1][k] : kd[0][k], idesc_s, k != 0);
-                tc::mma_commit(&s_full[t]);
-                tc::mma_commit(&k_empty[kb]);                   // one arrival per tile
-                if (last_of_item) tc::mma_commit(q_free);       // Q is no longer needed once this S has executed
+                for (int k = 0; k < KS; ++k) tc::mma_bf16_if(el, d_s, qd[k], kb ? kd[1][k] : kd[0][k], idesc_s, k != 0);
+                tc::mma_commit_if(el, &s_full[t]);
+                tc::mma_commit_if(el, &k_empty[kb]);            // one arrival per tile
+                if (last_of_item) tc::mma_commit_if(el, q_free);   // Q is no longer needed once this S has executed
             };
-            auto issue_o = [&](int vb, uint32_t accumulate) {   // O_t (+)= P_t V over the 128 keys in steps of 16
+            auto issue_o = [&](uint32_t el, int vb, uint32_t accumulate) {   // O_t (+)= P_t V over the 128 keys in steps of 16
 #pragma unroll
-                for (int k = 0; k < 8; ++k) tc::mma_bf16(d_o, pd[k], vb ? vd[1][k] : vd[0][k], idesc_o, (accumulate | (uint32_t)k) != 0 ? 1u : 0u);
-                tc::mma_commit(&o_full[t]);
-                tc::mma_commit(&v_empty[vb]);
+                for (int k = 0; k < 8; ++k) tc::mma_bf16_if(el, d_o, pd[k], vb ? vd[1][k] : vd[0][k], idesc_o, (accumulate | (uint32_t)k) != 0 ? 1u : 0u);
+                tc::mma_commit_if(el, &o_full[t]);
+                tc::mma_commit_if(el, &v_empty[vb]);
             };
             bool ok = total > 0 && wait2(bar_q, 0, bar_qz, 0) && wait(&k_full[0], 0);
             if (ok) {
                 tc::tc_fence_after();
-                if (tc::elect_one()) issue_s(0, nb == 1);
+                issue_s(tc::elect_one() ? 1u : 0u, 0, nb == 1);
                 __syncwarp();
             }
             int j = 0, it = 0;                                  // block within the item, item count
@@ -288,7 +289,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
                                 if (!ok) break;
                             }
                             tc::tc_fence_after();
-                            if (tc::elect_one()) issue_s(b ^ 1, new_item ? nb == 1 : j + 2 == nb);
+                            issue_s(tc::elect_one() ? 1u : 0u, b ^ 1, new_item ? nb == 1 : j + 2 == nb);
                             __syncwarp();
                         }
                     } else {
@@ -299,7 +300,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
                             if (!ok) break;
                         }
                         tc::tc_fence_after();
-                        if (tc::elect_one()) issue_o(b, j > 0 ? 1u : 0u);
+                        issue_o(tc::elect_one() ? 1u : 0u, b, j > 0 ? 1u : 0u);
                         __syncwarp();
                     }
                 }
