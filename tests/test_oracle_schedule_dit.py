@@ -280,3 +280,117 @@ def test_drafter_reuses_target_embedding_and_is_one_block():
     # the feature half of the fusion layer matters, and so does the latent half
     assert np.abs(drafter.forward(w, wd, sh, x, 0 * f, 12.0, 1)[1] - f_next).max() > 1e-3
     assert np.abs(drafter.forward(w, wd, sh, 0 * x, f, 12.0, 1)[1] - f_next).max() > 1e-3
+
+
+# ----------------------------------------------------------------------------- conditioning, head, whole forward, guided drafter
+_T = lambda a: torch.from_numpy(np.asarray(a, np.float64))
+
+
+def _torch_conditioning(w, sh, tau, label):
+    """c = W2 SiLU(W1 [cos, sin](tau w_i) + b1) + b2 + E[label], from torch functional ops only."""
+    half = sh.freq_dim // 2
+    ang = tau * torch.exp(-np.log(10000.0) * torch.arange(half, dtype=torch.float64) / half)
+    feat = torch.cat([torch.cos(ang), torch.sin(ang)])
+    e_t = F.linear(F.silu(F.linear(feat, _T(w["t_w1"]), _T(w["t_b1"]))), _T(w["t_w2"]), _T(w["t_b2"]))
+    return e_t + F.embedding(torch.tensor(label), _T(w["y_emb"]))
+
+
+def _torch_block(x, sc, w, i, h):
+    D = x.shape[1]
+    mod = F.linear(sc, _T(w["ada_w"][i]), _T(w["ada_b"][i])).chunk(6)
+    y = F.layer_norm(x, (D,), eps=1e-6) * (1 + mod[1]) + mod[0]
+    qkv = F.linear(y, _T(w["qkv_w"][i]), _T(w["qkv_b"][i])).reshape(-1, 3, h, D // h).permute(1, 2, 0, 3)
+    a = F.scaled_dot_product_attention(qkv[0][None], qkv[1][None], qkv[2][None])[0].permute(1, 0, 2).reshape(-1, D)
+    x = x + mod[2] * F.linear(a, _T(w["proj_w"][i]), _T(w["proj_b"][i]))
+    y = F.layer_norm(x, (D,), eps=1e-6) * (1 + mod[4]) + mod[3]
+    y = F.linear(F.gelu(F.linear(y, _T(w["fc1_w"][i]), _T(w["fc1_b"][i])), approximate="tanh"), _T(w["fc2_w"][i]), _T(w["fc2_b"][i]))
+    return x + mod[5] * y
+
+
+def _torch_head(x, sc, w, sh):
+    """Modulated head, then fold: token (i, j) holds (row-in-patch, column-in-patch, channel)."""
+    D, p, g = x.shape[1], sh.patch, sh.H // sh.patch
+    shift, scale = F.linear(sc, _T(w["fada_w"]), _T(w["fada_b"])).chunk(2)
+    tok = F.linear(F.layer_norm(x, (D,), eps=1e-6) * (1 + scale) + shift, _T(w["fin_w"]), _T(w["fin_b"]))
+    # F.fold wants [C*kh*kw, L] with the channel slowest: reorder (p, q, c) -> (c, p, q)
+    cols = tok.reshape(-1, p, p, sh.c_out).permute(3, 1, 2, 0).reshape(sh.c_out * p * p, g * g)
+    return F.fold(cols[None], (sh.H, sh.W), kernel_size=p, stride=p)[0]
+
+
+def test_conditioning_against_torch_functional_ops():
+    sh, w = _tiny(seed=3)
+    for tau, label in ((0.0, 0), (37.0, 4), (999.0, sh.n_classes)):         # the last one is the null-label row
+        ref = _torch_conditioning(w, sh, tau, label).numpy()
+        assert np.allclose(dit.conditioning(w, sh, tau, label), ref, rtol=0, atol=1e-13)
+    # the two timestep layers really have a SiLU between them, and the label row really is added
+    e = dit.conditioning(w, sh, 37.0, 4)
+    assert np.abs(e - dit.conditioning(w, sh, 37.0, 5)).max() > 1e-3
+    lin = dit.linear(dit.linear(dit.timestep_features(37.0, sh.freq_dim), w["t_w1"], w["t_b1"]), w["t_w2"], w["t_b2"])
+    assert np.abs(e - (lin + w["y_emb"][4])).max() > 1e-4
+
+
+def test_final_layer_against_torch_functional_ops():
+    sh, w = _tiny(seed=4, ada_std=0.3, out_gain=2.0)
+    rng = np.random.default_rng(8)
+    x, sc = rng.standard_normal((sh.n_tok, sh.D)) * 2 + 0.3, rng.standard_normal(sh.D)
+    got = dit.final_layer(x, sc, dit._with_heads(w, sh), sh)
+    ref = _torch_head(_T(x), _T(sc), w, sh).numpy()
+    assert got.shape == (sh.c_out, sh.H, sh.W) and np.allclose(got, ref, rtol=0, atol=1e-12)
+    # the pin can tell shift from scale and sees the LayerNorm: each planted variant is far outside the tolerance
+    D = sh.D
+    mod = dit.linear(sc, w["fada_w"], w["fada_b"])
+    swapped = dit.unpatchify(dit.linear(dit.layer_norm(x) * (1 + mod[:D]) + mod[D:], w["fin_w"], w["fin_b"]), sh)
+    no_one = dit.unpatchify(dit.linear(dit.layer_norm(x) * mod[D:] + mod[:D], w["fin_w"], w["fin_b"]), sh)
+    no_ln = dit.unpatchify(dit.linear(x * (1 + mod[D:]) + mod[:D], w["fin_w"], w["fin_b"]), sh)
+    for wrong in (swapped, no_one, no_ln):
+        assert np.abs(wrong - ref).max() > 1e-3
+
+
+@pytest.mark.parametrize("label", [2, 10])
+def test_whole_forward_against_torch_functional_ops(label):
+    # conditioning -> embed (strided convolution) -> blocks -> modulated head -> fold -> first C channels
+    sh, w = _tiny(seed=5, ada_std=0.3, out_gain=2.0)
+    x = synth.normal(5, 60, (sh.C, sh.H, sh.W)).astype(np.float64)
+    eps, feat = dit.forward(w, sh, x, 123.0, label)
+    sc = F.silu(_torch_conditioning(w, sh, 123.0, label))
+    h = F.conv2d(_T(x)[None], _T(w["pe_w"]).reshape(sh.D, sh.C, sh.patch, sh.patch), _T(w["pe_b"]), stride=sh.patch)[0]
+    h = h.flatten(1).T + _T(w["pos"])
+    for i in range(sh.depth):
+        h = _torch_block(h, sc, w, i, sh.heads)
+    out = _torch_head(h, sc, w, sh)
+    assert np.allclose(feat, h.numpy(), rtol=0, atol=1e-12)
+    assert eps.shape == (sh.C, sh.H, sh.W) and np.allclose(eps, out[:sh.C].numpy(), rtol=0, atol=1e-12)
+    assert np.abs(eps).max() > 1e-2                                         # not a comparison of zeros
+
+
+def test_guided_drafter_step_combines_two_streams_with_their_own_features():
+    sh, w = _tiny(seed=6, ada_std=0.3, out_gain=3.0)
+    wd = synth.make_drafter_weights(sh, 11, ada_std=0.3, out_gain=3.0)
+    sc = schedule.make("linear", 50)
+    rng = np.random.default_rng(12)
+    x = rng.standard_normal((sh.C, sh.H, sh.W))
+    f = rng.standard_normal((2, sh.n_tok, sh.D))
+    s, label, cfg = 17, 3, 4.0
+    m_hat, eps_hat, f_next = drafter.guided_step(w, wd, sh, sc, x, f, s, label, cfg)
+    tau = sc.t_embed_value[s]
+    e_c, f_c = drafter.forward(w, wd, sh, x, f[0], tau, label)               # conditional stream: label, its own feature
+    e_u, f_u = drafter.forward(w, wd, sh, x, f[1], tau, sh.n_classes)        # unconditional stream: null label, its own feature
+    eps_ref = e_u + cfg * (e_c - e_u)
+    assert np.allclose(eps_hat, eps_ref, rtol=0, atol=1e-14)
+    assert np.array_equal(f_next[0], f_c) and np.array_equal(f_next[1], f_u)
+    assert np.allclose(m_hat, sc.coef_x[s] * x - sc.coef_eps[s] * eps_ref, rtol=0, atol=1e-13)   # Eq. ddpm_update
+    assert np.allclose(m_hat, (x - sc.betas[s] / np.sqrt(1 - sc.abar[s]) * eps_ref) / np.sqrt(sc.alphas[s]), atol=1e-12)
+    # swapping the two streams' features, guiding the other way round, or guiding the mean instead of the noise are all visible
+    swapped = drafter.guided_step(w, wd, sh, sc, x, f[::-1], s, label, cfg)
+    assert np.abs(swapped[1] - eps_hat).max() > 1e-3 and np.abs(swapped[2][0] - f_next[0]).max() > 1e-3
+    assert np.abs((e_c + cfg * (e_u - e_c)) - eps_hat).max() > 1e-3
+    # guidance off: one stream only, and the unconditional feature is not consulted
+    m1, e1, f1 = drafter.guided_step(w, wd, sh, sc, x, f, s, label, 1.0)
+    assert np.array_equal(e1, e_c) and f1.shape == (1, sh.n_tok, sh.D)
+    # the drafter's whole forward against torch functional ops: fuse -> one block -> its own head
+    g = F.linear(torch.cat([F.conv2d(_T(x)[None], _T(w["pe_w"]).reshape(sh.D, sh.C, sh.patch, sh.patch), _T(w["pe_b"]),
+                                     stride=sh.patch)[0].flatten(1).T + _T(w["pos"]), _T(f[0])], dim=1), _T(wd["fc_w"]), _T(wd["fc_b"]))
+    scc = F.silu(_torch_conditioning(w, sh, float(tau), label))
+    hh = _torch_block(g, scc, wd, 0, sh.heads)
+    assert np.allclose(f_c, hh.numpy(), atol=1e-12)
+    assert np.allclose(e_c, _torch_head(hh, scc, wd, sh)[:sh.C].numpy(), atol=1e-12)
