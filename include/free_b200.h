@@ -100,6 +100,37 @@ typedef struct free_schedule {
     const float* t_embed_value;
 } free_schedule;
 
+/*
+ * free_schedule_linear / free_schedule_respaced -- the reverse-process tables of a DDPM noise schedule, in fp64,
+ * HOST-only (no CUDA call; any thread).  The caller rounds them to fp32 and uploads them for `free_schedule`.
+ *   beta_s linear from beta_first (s = 0) to beta_last (s = N-1); alpha_s = 1 - beta_s; abar_s = prod_{r<=s} alpha_r.
+ *   Reverse step of Eq. ddpm_update (Appendix "Variance Setting"):
+ *       coef_x[s] = 1 / sqrt(alpha_s),   coef_eps[s] = beta_s / (sqrt(1 - abar_s) sqrt(alpha_s)).
+ *   variance_mode selects the fixed variance (the Appendix allows any predefined sigma_t):
+ *       FREE_VAR_POSTERIOR  sigma2 = beta~_s = beta_s (1 - abar_{s-1}) / (1 - abar_s), abar_{-1} = 1   (Sec. 4)
+ *       FREE_VAR_BETA       sigma2 = beta_s
+ *       FREE_VAR_INTERP     sigma2 = beta_s^v beta~_s^(1-v), v = variance_weight in [0, 1]
+ *   stochasticity >= 0 replaces the step by one Euler-Maruyama step of the epsilon-family of reverse processes
+ *   (Appendix "Stochasticity Hyperparameter", Eq. mean_var_gamma) for the variance-preserving process, with
+ *   e = stochasticity:  coef_x = 1 + beta_s / 2,  coef_eps = (1 + e^2)/2 beta_s / sqrt(1 - abar_s),
+ *   sigma2 = e^2 beta_s  (variance_mode is then ignored).  Pass a negative value for the DDPM step above.
+ *   In every variant sigma2[0] = 0: the last transition adds no noise.
+ *   free_schedule_respaced keeps abar of the n_full-step linear schedule at the N evenly spaced indices
+ *   round_half_even(i (n_full-1)/(N-1)), recomputes beta from consecutive ratios of abar, and reports those original
+ *   indices in t_embed_value (what the timestep embedder sees); free_schedule_linear reports s itself.
+ *   coef_x, coef_eps, sigma2, t_embed_value   HOST double [N], written
+ * Errors: ARG (null pointer, bad mode), SHAPE (N < 2, n_full < N, betas outside (0, 1), weight outside [0, 1]).
+ */
+#define FREE_VAR_POSTERIOR 0
+#define FREE_VAR_BETA      1
+#define FREE_VAR_INTERP    2
+int free_schedule_linear(int N, double beta_first, double beta_last,
+                         int variance_mode, double variance_weight, double stochasticity,
+                         double* coef_x, double* coef_eps, double* sigma2, double* t_embed_value);
+int free_schedule_respaced(int N, int n_full, double beta_first, double beta_last,
+                           int variance_mode, double variance_weight, double stochasticity,
+                           double* coef_x, double* coef_eps, double* sigma2, double* t_embed_value);
+
 typedef struct free_ctx free_ctx;
 
 /* Validate the descriptors, record them (weights are NOT copied: they must outlive the context) and

@@ -86,6 +86,8 @@ _SIGNATURES = {
     "free_uncertainty_profile": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.POINTER(ScheduleDesc),
                                            C.POINTER(SpecParams), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "free_schedule_linear": (C.c_int, [C.c_int, C.c_double, C.c_double, C.c_int, C.c_double, C.c_double] + [C.c_void_p] * 4),
+    "free_schedule_respaced": (C.c_int, [C.c_int, C.c_int, C.c_double, C.c_double, C.c_int, C.c_double, C.c_double] + [C.c_void_p] * 4),
     "free_fit_lambda_profile": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p]),
     "free_drafter_loss_workspace_bytes": (C.c_size_t, []),
     "free_drafter_loss": (C.c_int, [C.c_int] * 4 + [C.c_int64] + [C.c_void_p] * 4 + [C.c_float] * 4 +

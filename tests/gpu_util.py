@@ -14,6 +14,14 @@ def nerr(got, ref):
     return float(np.abs(got.astype(np.float64).reshape(ref.shape) - ref).max() / max(np.abs(ref).max(), 1e-30))
 
 
+def rms_rel(got, ref):
+    """sqrt(mean (got - ref)^2) / sqrt(mean ref^2): unlike `nerr` it sees an error confined to small elements."""
+    got = got.detach().float().cpu().numpy() if isinstance(got, torch.Tensor) else np.asarray(got)
+    ref = np.asarray(ref, np.float64)
+    diff = got.astype(np.float64).reshape(ref.shape) - ref
+    return float(np.sqrt(np.mean(diff * diff)) / max(np.sqrt(np.mean(ref * ref)), 1e-30))
+
+
 def round_by_hand(free, model, sh, dsched, tables, x_cur, cursor, labels, K, cfg, zt, zd, u):
     """One round of Algorithm 1 assembled from the public calls (target step, K drafter steps, raw packed pass, fused
     verifier) for samples whose cursor leaves room for all K drafts.  x_cur [B,C,H,W], cursor [B] (1-based next

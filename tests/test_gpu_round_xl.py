@@ -6,10 +6,16 @@ import torch
 
 import synth
 from oracle import dit as odit, schedule as osched
-from gpu_util import cu, nerr
+from gpu_util import cu, nerr, rms_rel
 
 pytestmark = pytest.mark.gpu
 TOL = 2e-2
+# RMS-relative bound.  A bf16 rounding has relative RMS error 2^-9/sqrt(3) = 1.1e-3.  A block rounds four GEMM operands
+# (modulated LayerNorm output twice, attention output, MLP hidden) plus q/k/v and P; the branch outputs enter the fp32
+# residual stream through gates of RMS ~ 0.1 * |SiLU(c)| and are renormalised by the next LayerNorm, so the relative
+# error of the stream grows like a random walk over 28 x ~6 roundings: 1.1e-3 * sqrt(168) = 1.5e-2 if every rounding
+# came through at full weight.  The gates pass well under half of it; 1e-2 leaves that margin and is half of TOL.
+TOL_RMS = 1e-2
 
 
 @pytest.fixture(scope="module")
@@ -33,11 +39,15 @@ def test_xl_512_packed_pass_sampled_against_oracle(xl):
     torch.cuda.synchronize()
     assert model.device_error() == 0
     assert torch.isfinite(mean).all() and torch.isfinite(feat.float()).all()
-    pick = [37]                                  # one state = two full-depth sequences of the oracle
-    mo, eo, fo = odit.verify_pass(w, sh, sc, X[pick], T[pick], Y[pick], 4.0)
-    errs = (nerr(eps[pick], eo), nerr(mean[pick], mo), nerr(feat[pick], fo))
-    print("XL/2 512 errors eps/mean/feat:", errs)
-    assert max(errs) < TOL
+    pick = [0, 37, 62, 95]                       # first, last and two interior states (different samples, timesteps and
+    mo, eo, fo = odit.verify_pass(w, sh, sc, X[pick], T[pick], Y[pick], 4.0)     # labels): 8 full-depth oracle sequences
+    assert len(set(T[pick].tolist())) == 4 and len(set(Y[pick].tolist())) == 4
+    for i, st in enumerate(pick):
+        errs = (nerr(eps[st], eo[i]), nerr(mean[st], mo[i]), nerr(feat[st], fo[i]))
+        rms = (rms_rel(eps[st], eo[i]), rms_rel(mean[st], mo[i]), rms_rel(feat[st], fo[i]))
+        print("XL/2 512 state %d: max-normalised eps/mean/feat %s  RMS-relative %s" % (st, errs, rms))
+        assert max(errs) < TOL and max(rms) < TOL_RMS
+    pick = [37]
     # batch invariance at full size: the same state alone gives the same result
     one = model.dit_verify_pass(cu(X[pick]), cu(T[pick], torch.int32), cu(Y[pick], torch.int32), 4.0, dsched)
     assert nerr(one, mean[pick].cpu().numpy()) < 1e-6
@@ -59,8 +69,16 @@ def test_xl_round_consistency(xl):
     assert n1.tolist() == [6, 4] and c1.tolist() == [28, 250]     # u = 0: every draft accepted
     x2, c2, n2 = model.spec_round(x0, cursor, labels, dsched, K, 4.0, zt, zd, cu(np.ones((B, N), np.float32)))
     torch.cuda.synchronize()
-    assert all(a <= 1 for a in n2.tolist()) or True
+    # u = 1 accepts a draft only where its log-ratio is >= 0.  Whatever the counts are, the cursor moves past the
+    # accepted drafts and the reflected one, and never past the drafts that exist (6 and 4)
+    nv = np.array([6, 4])
+    n2, c2 = n2.cpu().numpy(), c2.cpu().numpy()
+    assert np.all(n2 >= 0) and np.all(n2 <= nv)
+    assert np.array_equal(c2, cursor.cpu().numpy() + 1 + np.minimum(n2 + 1, nv))
     assert torch.isfinite(x1).all() and torch.isfinite(x2).all()
+    for b in range(B):                           # a sample that stopped early ends on a reflected state, not on the last draft
+        if n2[b] < nv[b]:
+            assert not torch.equal(x1[b], x2[b])
 
 
 def test_xl_round_teacher_forced(xl):
@@ -88,6 +106,8 @@ def test_xl_256_packed_pass_sampled_against_oracle():
     assert model.device_error() == 0
     pick = [0, 41]
     mo, eo, fo = odit.verify_pass(w, sh, sc, X[pick], T[pick], Y[pick], 4.0)
-    errs = (nerr(eps[pick], eo), nerr(mean[pick], mo), nerr(feat[pick], fo))
-    print("XL/2 256 errors eps/mean/feat:", errs)
-    assert max(errs) < TOL
+    for i, st in enumerate(pick):
+        errs = (nerr(eps[st], eo[i]), nerr(mean[st], mo[i]), nerr(feat[st], fo[i]))
+        rms = (rms_rel(eps[st], eo[i]), rms_rel(mean[st], mo[i]), rms_rel(feat[st], fo[i]))
+        print("XL/2 256 state %d: max-normalised eps/mean/feat %s  RMS-relative %s" % (st, errs, rms))
+        assert max(errs) < TOL and max(rms) < TOL_RMS

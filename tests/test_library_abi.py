@@ -58,3 +58,35 @@ def test_argument_errors_need_no_gpu(libpath):
     q = ctypes.c_void_p(4100)
     assert L.spec_verify(1, 4, 16, q, p, p, p, None, p, None, p, p, None, None) == -3     # misaligned
     assert L.spec_verify(0, 4, 16, p, p, p, p, None, p, None, p, p, None, None) == 0      # empty batch
+
+
+def test_schedule_constructors_errors_and_closed_forms(libpath):
+    # the library's host-side schedule constructors: argument errors, and values that follow from the definitions
+    import numpy as np
+    from paper_2511_20390_b200 import binding, linear_schedule, respaced_schedule
+    L = binding.lib()
+    buf = [np.empty(8) for _ in range(4)]
+    ptr = [a.ctypes.data_as(ctypes.c_void_p) for a in buf]
+    assert L.free_schedule_linear(8, 1e-4, 2e-2, 0, 0.0, -1.0, None, *ptr[1:]) == -1          # null table
+    assert L.free_schedule_linear(8, 1e-4, 2e-2, 7, 0.0, -1.0, *ptr) == -1                     # unknown variance mode
+    assert L.free_schedule_linear(1, 1e-4, 2e-2, 0, 0.0, -1.0, *ptr) == -2                     # N < 2
+    assert L.free_schedule_linear(8, 0.0, 2e-2, 0, 0.0, -1.0, *ptr) == -2                      # beta must lie in (0, 1)
+    assert L.free_schedule_linear(8, 1e-4, 1.5, 0, 0.0, -1.0, *ptr) == -2
+    assert L.free_schedule_linear(8, 1e-4, 2e-2, 2, 1.5, -1.0, *ptr) == -2                     # interpolation weight outside [0, 1]
+    assert L.free_schedule_respaced(8, 4, 1e-4, 2e-2, 0, 0.0, -1.0, *ptr) == -2                # fewer original steps than kept
+    assert L.free_schedule_linear(8, 1e-4, 2e-2, 0, 0.0, -1.0, *ptr) == 0
+    with pytest.raises(ValueError):
+        linear_schedule(8, variance=1.5)
+    # two-step schedule by hand: alpha = (1-b0, 1-b1); sigma2 = (0, b1 b0 / (1 - a0 a1))
+    b0, b1 = 0.1, 0.3
+    t = linear_schedule(2, b0, b1)
+    assert np.allclose(t["coef_x"], [1 / np.sqrt(0.9), 1 / np.sqrt(0.7)], rtol=1e-15)
+    assert np.allclose(t["coef_eps"], [b0 / np.sqrt(b0 * 0.9), b1 / np.sqrt((1 - 0.63) * 0.7)], rtol=1e-15)
+    assert t["sigma2"][0] == 0.0 and np.isclose(t["sigma2"][1], b1 * b0 / (1 - 0.63), rtol=1e-15)
+    assert np.array_equal(t["t_embed_value"], [0.0, 1.0])
+    # keeping every step of the full schedule changes nothing; the kept indices of 1000 -> 250 are 4 or 5 apart
+    full, same = linear_schedule(50), respaced_schedule(50, 50)
+    for k in full:
+        assert np.allclose(full[k], same[k], rtol=1e-12, atol=1e-300)
+    keep = respaced_schedule(250)["t_embed_value"]
+    assert keep[0] == 0 and keep[-1] == 999 and set(np.diff(keep)) <= {4.0, 5.0}
