@@ -357,6 +357,22 @@ int free_profile_begin(free_ctx* ctx);
 int free_profile_end(free_ctx* ctx, free_prof_entry* out, int max_entries, int* n_entries);
 
 /*
+ * Device error word (safety aid; the paper has no counterpart).  free_device_error_code() maps a HOST copy of a device
+ * error word to the library's return code: 0 -> FREE_OK, anything else -> FREE_ERR_DEVICE_TIMEOUT.  It is the mapping
+ * sample_trajectory() applies after every round.
+ * free_selftest_bounded_wait() runs the bounded wait of the tensor-core pipelines once on a barrier that nothing ever
+ * signals: one warp, no copies, tensor memory or clusters involved.  The wait gives up after `limit_cycles` SM clock
+ * cycles (1 .. 1e8, i.e. at most about 50 ms), ORs a non-zero code into *device_error exactly as the pipelines do, and
+ * the kernel returns; the context stays usable.  It shows that an expired wait ends in an error status, not in a stuck
+ * launch.
+ *   device_error   DEVICE uint32, OR-ed into (clear it first)
+ *   waited_cycles  DEVICE int64 or NULL: SM cycles the wait took
+ * Asynchronous.  Errors: ARG, SHAPE (limit out of range), ALIGN, CUDA.
+ */
+int free_device_error_code(uint32_t word);
+int free_selftest_bounded_wait(uint32_t* device_error, int64_t limit_cycles, int64_t* waited_cycles, void* stream);
+
+/*
  * free_drafter_loss -- the drafter's training objectives (Sec. 3.2), forward values, as one fused reduction:
  *   L_noise  = mean over all elements of (eps_pred - eps_ref)^2                                   (Eq. mse)
  *   L_feat   = mean over sequences and tokens of 1 - <p, r> / (|p| |r| + eps_cos)                 (Eq. cos)

@@ -92,6 +92,8 @@ _SIGNATURES = {
     "free_drafter_loss_workspace_bytes": (C.c_size_t, []),
     "free_drafter_loss": (C.c_int, [C.c_int] * 4 + [C.c_int64] + [C.c_void_p] * 4 + [C.c_float] * 4 +
                           [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "free_device_error_code": (C.c_int, [C.c_uint32]),
+    "free_selftest_bounded_wait": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]),
     "free_profile_begin": (C.c_int, [C.c_void_p]),
     "free_profile_end": (C.c_int, [C.c_void_p, C.POINTER(ProfEntry), C.c_int, C.POINTER(C.c_int)]),
     "free_op_linear_workspace_bytes": (C.c_size_t, []),
@@ -272,6 +274,17 @@ def spec_verify_host(m, m_hat, x_hat, sigma2, u, lam=None):
 # ------------------------------------------------------------------------------------------ model
 _ACT = {FREE_FP32: torch.float32, FREE_BF16: torch.bfloat16}
 _MATRICES = ("t_w1", "t_w2", "ada_w", "qkv_w", "proj_w", "fc1_w", "fc2_w", "fada_w", "fc_w")
+
+
+def selftest_bounded_wait(limit_cycles: int = 100_000):
+    """Runs the pipelines' bounded wait once on a barrier nothing signals (free_selftest_bounded_wait).  Returns
+    (error word, SM cycles waited, library return code the word maps to)."""
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    waited = torch.zeros(1, dtype=torch.int64, device="cuda")
+    _check(lib().free_selftest_bounded_wait(_ptr(err), int(limit_cycles), _ptr(waited), _stream()), "free_selftest_bounded_wait")
+    torch.cuda.current_stream().synchronize()
+    word = int(err.item()) & 0xFFFFFFFF
+    return word, int(waited.item()), int(lib().free_device_error_code(word))
 
 
 class DeviceSchedule:

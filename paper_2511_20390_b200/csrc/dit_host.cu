@@ -691,7 +691,7 @@ int run_trajectory(free_ctx* c, int B, const float* x0, const int32_t* labels, c
         uint32_t dev_err = 0;
         FREE_CUDA_TRY(cudaMemcpyAsync(&dev_err, w.err, 4, cudaMemcpyDeviceToHost, s));
         FREE_CUDA_TRY(cudaStreamSynchronize(s));
-        if (dev_err) return FREE_ERR_DEVICE_TIMEOUT;
+        FREE_TRY(free_device_error_code(dev_err));
         for (int b = 0; b < B; ++b) {
             if (!h_act[b]) continue;
             if (K > 0 && h_nv[b] > 0 && h_acc[b] < 0) return h_acc[b];
