@@ -1,10 +1,12 @@
 """Benchmark of the packed parallel-verification path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload round|verifier|verifier_fused|drafter_loss|trajectory] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload round|verifier|verifier_fused|verifier_sweep|drafter_loss|trajectory|ops] [--impl reference]
 
 One JSON line on stdout (rank 0).  A "step" is one pass of the hot path over one batch of synthetic
 input resident in HBM; `e2e` repeats it from pinned HOST buffers with the copies inside the timed
-region.  `--impl reference` times the CPU oracle on a bounded sample of the same workload.
+region.  The default workload (one FREE round on the DiT-XL/2-shaped 512^2 model) also reports, from the same
+process, the verifier on its own (`verifier_roofline`) and whole trajectories in images/s (`trajectory`), and takes its
+per-kernel table in a second pass so that the headline is timed without per-launch events.  `--impl reference` times the CPU oracle on a bounded sample of the same workload.
 Multi-GPU runs shard whole batches across ranks (weak scaling, no data-path collective).
 """
 import argparse
@@ -33,6 +35,8 @@ def parse():
     ap.add_argument("--res", type=int, default=512, choices=[256, 512], help="trajectory workload: image resolution")
     ap.add_argument("--chunk", type=int, default=0, help="verifier_fused: drafts per early-exit chunk (0 = off)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="default workload: skip the verifier and trajectory measurements")
+    ap.add_argument("--K", type=int, default=0, help="verifier workloads: drafts per sample (0 = 16)")
     return ap.parse_args()
 
 
@@ -322,6 +326,69 @@ def make_workload(name, batch, rank, chunk=0):
     raise SystemExit(f"unknown workload {name}")
 
 
+def time_launches(fn, launches=20, warm=3):
+    """Mean device time (ms) of `launches` calls of fn on the current stream, CUDA events, after `warm` calls."""
+    import torch
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(launches):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / launches
+
+
+def verifier_extras(peaks, launches=20):
+    """The verifier on its own at the largest point of the sweep (K = 16, B = 256, latent 4x64x64; inputs of 0.8 / 1.1 GB,
+    larger than L2): from means (spec_verify) and from the noise predictions (spec_verify_fused)."""
+    import gc
+    import torch
+    out = {}
+    for key, cls in (("standalone", VerifierWorkload), ("fused", FusedVerifierWorkload)):
+        wl = cls(0, 0)
+        ms = time_launches(wl.step, launches)
+        r = wl.roofline(ms, peaks)
+        out[key] = {"kernel": r["kernel"], "bound": "hbm", "achieved": r["achieved"], "peak": r["peak"], "unit": "GB/s", "frac": r["frac"],
+                    "traffic": r["traffic"], "ms_per_launch": ms, "launches": launches, "bytes_per_launch": wl.bytes_per_step,
+                    "workload": wl.name}
+        del wl
+        gc.collect(); torch.cuda.empty_cache()
+    out["peak_source"] = peaks["source"] + " (copy bandwidth)"
+    return out
+
+
+def verifier_sweep(args, peaks):
+    """`--workload verifier_sweep`: GB/s and fraction of the measured copy bandwidth of spec_verify over the sweep of
+    drafts per sample, batch and acceptance mode (latent 4x64x64).  Points whose inputs fit L2 are marked: their figure is
+    a cache figure, not an HBM one."""
+    import torch
+    import synth
+    import paper_2511_20390_b200 as free
+    d = 16384
+    sched = free.respaced_schedule(250)
+    rows = []
+    for K in ([args.K] if args.K else [2, 4, 6, 8, 16]):
+        for B in ([args.batch] if args.batch else [1, 4, 16, 64, 256]):
+            s2 = np.tile(sched["sigma2"][np.linspace(240, 20, K).astype(int)].astype(np.float32), (B, 1))
+            m, mh, xh, u = synth.verifier_inputs(4000 + K, B, K, d, 0.0015, s2)
+            dev = [torch.from_numpy(a).cuda() for a in (m, mh, xh, s2, u)]
+            lam = torch.full((B, K), 0.5, device="cuda")
+            x_out, n_acc = torch.empty(B, d, device="cuda"), torch.empty(B, dtype=torch.int32, device="cuda")
+            by = B * (3 * K * d * 4 + d * 4 + 12 * K)
+            for mode, lm in (("strict", None), ("relaxed", lam)):
+                ms = time_launches(lambda: free.spec_verify(*dev, lam=lm, x_out=x_out, n_accept=n_acc), 20)
+                gbs = by / 1e9 / (ms / 1e3)
+                rows.append({"K": K, "B": B, "mode": mode, "us": round(ms * 1e3, 2), "gbs": round(gbs, 1),
+                             "frac_of_copy": round(gbs / peaks["hbm_gbs"], 4), "MB": round(by / 1e6, 2),
+                             "fits_l2": by < 126e6})
+    print(json.dumps({"metric": "verifier HBM GB/s", "unit": "GB/s", "peak": peaks["hbm_gbs"], "peak_source": peaks["source"],
+                      "config": {"workload": "spec_verify sweep, latent 4x64x64, 20 launches per point after 3 warm-ups"},
+                      "points": rows}))
+
+
 def max_over_ranks(times_ms, device):
     """Element-wise maximum of per-rank timings over all ranks (every rank gets the result); single process: identity.
     The job's time is that of its slowest rank."""
@@ -407,8 +474,12 @@ def main():
             run_trajectory(args)
         return
 
-    wl = make_workload(args.workload, args.batch, rank, args.chunk)
     peaks = measured_peaks()
+    if args.workload == "verifier_sweep":
+        if rank == 0:
+            verifier_sweep(args, peaks)
+        return
+    wl = make_workload(args.workload, args.batch, rank, args.chunk)
 
     def barrier():
         if world > 1:
@@ -421,16 +492,20 @@ def main():
     sampler = ClockSampler(local_rank) if rank == 0 else None
     stream = torch.cuda.current_stream()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    if hasattr(wl, "begin_timed"):
-        wl.begin_timed()          # per-kernel CUDA events on the launching stream, inside the timed region
     ev0.record(stream)
     for _ in range(args.steps):
         wl.step()
     ev1.record(stream)
     barrier()
     ms = ev0.elapsed_time(ev1)
-    if hasattr(wl, "end_timed"):
+    if hasattr(wl, "begin_timed"):
+        # second pass of the same steps with CUDA events around every kernel launch (the per-kernel table and the
+        # roofline of the dominant kernel); the headline above is timed without them
+        wl.begin_timed()
+        for _ in range(args.steps):
+            wl.step()
         wl.end_timed(args.steps)
+        barrier()
     kernel_ms = wl.kernel_ms_per_launch() if hasattr(wl, "kernel_ms_per_launch") else ms / args.steps
     clocks = sampler.stop() if sampler else None
 
@@ -462,6 +537,11 @@ def main():
                "roofline": wl.roofline(kernel_ms, peaks)}
         if hasattr(wl, "extra"):
             out.update(wl.extra(ms_step, dict(peaks, sm_mhz=clocks["sm_mhz"] if clocks else None)))
+        if world == 1 and args.workload == "default" and not args.no_extras:
+            # the other two parts of the metric, measured in this process: verifier HBM GB/s and images/s
+            if hasattr(wl, "trajectory_extras"):
+                out["trajectory"] = wl.trajectory_extras()
+            out["verifier_roofline"] = verifier_extras(peaks)
         if world == 1 and not args.no_cpu_baseline:
             v, sample = wl.oracle_sample()
             out["cpu_baseline"] = {"value": v, "unit": wl.unit, "cores": cpu_threads(), "kind": "oracle", "sample": sample}

@@ -63,9 +63,16 @@ class RoundWorkload:
         self.flops = round_flops(sh, B, K, self.G)
         self.units_per_step = self.flops / 1e12
         self.config = round_config(B, K, self.G)
-        # host staging for the end-to-end path
+        # host staging for the end-to-end path: everything one round consumes.  From cursor a = 21 the round takes the
+        # target's noise of transition 21 (row 20), the drafter's noise of transitions 22..27 (rows 21..26) and the
+        # uniforms of the same six transitions
         pin = lambda t: torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t)
+        a0 = 20
+        self.rows_t, self.rows_d = slice(a0, a0 + 1), slice(a0 + 1, a0 + 1 + K)
         self.h_in = [pin(self.x_cur), pin(self.cursor), pin(self.labels)]
+        self.h_zt = [pin(self.noise_t[b, self.rows_t]) for b in range(B)]
+        self.h_zd = [pin(self.noise_d[b, self.rows_d]) for b in range(B)]
+        self.h_u = pin(self.uniforms)                  # [B, N] is 16 KB: the whole table travels
         self.h_out = [torch.empty(self.x_next.shape, dtype=torch.float32, pin_memory=True),
                       torch.empty(B, dtype=torch.int32, pin_memory=True), torch.empty(B, dtype=torch.int32, pin_memory=True)]
         self.launches_per_step = None
@@ -89,15 +96,18 @@ class RoundWorkload:
         self._round()
 
     def host_step(self):
-        t = self.torch
         self.x_cur.copy_(self.h_in[0], non_blocking=True)
         self.cursor.copy_(self.h_in[1], non_blocking=True)
         self.labels.copy_(self.h_in[2], non_blocking=True)
+        for b in range(self.B):                        # contiguous row runs: one plain asynchronous copy each
+            self.noise_t[b, self.rows_t].copy_(self.h_zt[b], non_blocking=True)
+            self.noise_d[b, self.rows_d].copy_(self.h_zd[b], non_blocking=True)
+        self.uniforms.copy_(self.h_u, non_blocking=True)
         self._round()
         self.h_out[0].copy_(self.x_next, non_blocking=True)
         self.h_out[1].copy_(self.cursor_next, non_blocking=True)
         self.h_out[2].copy_(self.n_acc, non_blocking=True)
-        h2d = sum(x.numel() * x.element_size() for x in self.h_in)
+        h2d = sum(x.numel() * x.element_size() for x in self.h_in + self.h_zt + self.h_zd + [self.h_u])
         d2h = sum(x.numel() * x.element_size() for x in self.h_out)
         return h2d, d2h
 
@@ -153,6 +163,13 @@ class RoundWorkload:
                                      "of_measured_burst": value / peaks["bf16_tflops"], "of_nominal_2250": value / 2250.0},
                 "images_per_s_if_all_accepted": self.B * (K_DRAFTS + 1) / N_SCHED / (ms_step / 1e3),
                 "kernels": kern}
+
+    def trajectory_extras(self):
+        """images/s of whole 250-transition trajectories with this workload's model and batch: every draft accepted
+        (u = 0: the most a round can finalise) and the sequential sampler (K = 0) on the same GPU."""
+        out = time_trajectories(self.model, self.shape, self.B, {"all_accepted": (K_DRAFTS, 0.0), "sequential_K0": (0, None)}, warm=False)
+        return {"unit": "images/s", "api": "sample_trajectory", "transitions": N_SCHED, "batch": self.B, "K": K_DRAFTS,
+                "timing": "CUDA events around the blocking call (one host synchronisation per round inside)", **out}
 
     def oracle_sample(self):
         return oracle_dit_sample(self.shape)
@@ -244,6 +261,47 @@ class OpsWorkload:
         return oracle_dit_sample(synth.DIT_XL2_512, 1)
 
 
+def time_trajectories(model, sh, B, regimes, seed=7, use_graph=False, warm=True):
+    """Whole sampling trajectories through sample_trajectory (Algorithm 1 end to end; the call blocks and synchronises
+    once per round): device time by CUDA events around each call.  `regimes`: name -> (K, uniforms or a constant or None)."""
+    import torch
+    import paper_2511_20390_b200 as free
+    sched = free.DeviceSchedule(free.respaced_schedule(N_SCHED))
+    g = torch.Generator(device="cuda"); g.manual_seed(seed)
+    d = sh.d_latent
+    rn = lambda *s_: torch.randn(*s_, generator=g, device="cuda", dtype=torch.float32)
+    x0 = rn(B, sh.C, sh.H, sh.W)
+    labels = torch.randint(0, sh.n_classes, (B,), generator=g, device="cuda", dtype=torch.int32)
+    zt, zd = rn(B, N_SCHED, d), rn(B, N_SCHED, d)
+    uni = {}
+    for name, (K, u) in regimes.items():
+        if u == "seeded":
+            u = torch.rand(B, N_SCHED, generator=g, device="cuda")
+        elif u is not None:
+            u = torch.full((B, N_SCHED), float(u), device="cuda")
+        uni[name] = u
+    if warm:
+        model.sample_trajectory(x0, labels, sched, K_DRAFTS, CFG, zt, zd, torch.zeros(B, N_SCHED, device="cuda"))
+        torch.cuda.synchronize()
+    out = {}
+    side = torch.cuda.Stream()            # the legacy default stream cannot be captured into a graph
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for name, (K, _) in regimes.items():
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            x, st = model.sample_trajectory(x0, labels, sched, K, CFG, zt, zd if K else None, uni[name], use_graph=use_graph)
+            e1.record()
+            torch.cuda.synchronize()
+            sec = e0.elapsed_time(e1) / 1e3
+            assert torch.isfinite(x).all()
+            out[name] = {"images_per_s": B / sec, "seconds": sec, "rounds": st["rounds"], "target_calls": st["target_calls"],
+                         "draft_calls": st["draft_calls"], "accepted": st["accepted"], "rejected": st["rejected"],
+                         "parallel_efficiency": st["parallel_efficiency"], "graph_rounds": st["graph_rounds"]}
+    torch.cuda.current_stream().wait_stream(side)
+    return out
+
+
 def run_trajectory(args):
     """`bench.py --workload trajectory`: whole sampling trajectories (Algorithm 1 end to end through sample_trajectory)
     on the DiT-XL/2-shaped 512^2 (or, with --res 256, 256^2) model, 250 transitions, guidance, batch B: images per second for the two bounding
@@ -259,34 +317,9 @@ def run_trajectory(args):
     sh = synth.DIT_XL2_256 if res == 256 else synth.DIT_XL2_512
     B = args.batch or 16
     model = free.Model.random(sh, 1234, dtype="bf16", with_drafter=True)
-    sched = free.DeviceSchedule(free.respaced_schedule(N_SCHED))
-    g = torch.Generator(device="cuda"); g.manual_seed(7)
-    d = sh.d_latent
-    rn = lambda *s_: torch.randn(*s_, generator=g, device="cuda", dtype=torch.float32)
-    x0 = rn(B, sh.C, sh.H, sh.W)
-    labels = torch.randint(0, sh.n_classes, (B,), generator=g, device="cuda", dtype=torch.int32)
-    zt, zd = rn(B, N_SCHED, d), rn(B, N_SCHED, d)
-    regimes = {"all_accepted": (K_DRAFTS, torch.zeros(B, N_SCHED, device="cuda")),
-               "almost_all_rejected": (K_DRAFTS, torch.ones(B, N_SCHED, device="cuda")),
-               "seeded_uniforms": (K_DRAFTS, torch.rand(B, N_SCHED, generator=g, device="cuda")),
-               "sequential_K0": (0, None)}
-    model.sample_trajectory(x0, labels, sched, K_DRAFTS, CFG, zt, zd, regimes["all_accepted"][1])      # warm-up
-    torch.cuda.synchronize()
-    out = {}
-    side = torch.cuda.Stream()            # the legacy default stream cannot be captured into a graph
-    side.wait_stream(torch.cuda.current_stream())
-    with torch.cuda.stream(side):
-        for name, (K, u) in regimes.items():
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            x, st = model.sample_trajectory(x0, labels, sched, K, CFG, zt, zd if K else None, u, use_graph=getattr(args, "graph", False))
-            e1.record()
-            torch.cuda.synchronize()
-            sec = e0.elapsed_time(e1) / 1e3
-            assert torch.isfinite(x).all()
-            out[name] = {"images_per_s": B / sec, "seconds": sec, "rounds": st["rounds"], "target_calls": st["target_calls"],
-                         "draft_calls": st["draft_calls"], "accepted": st["accepted"], "rejected": st["rejected"],
-                         "parallel_efficiency": st["parallel_efficiency"], "graph_rounds": st["graph_rounds"]}
+    regimes = {"all_accepted": (K_DRAFTS, 0.0), "almost_all_rejected": (K_DRAFTS, 1.0),
+               "seeded_uniforms": (K_DRAFTS, "seeded"), "sequential_K0": (0, None)}
+    out = time_trajectories(model, sh, B, regimes, use_graph=getattr(args, "graph", False))
     line = {"metric": "images/s", "value": out["all_accepted"]["images_per_s"], "unit": "images/s", "n_gpus": 1,
             "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": f"sample_trajectory, DiT-XL/2-shaped {res}^2, {N_SCHED} transitions, K={K_DRAFTS}, cfg {CFG}, batch {B}"

@@ -38,9 +38,23 @@ def test_bench_line(args, bound):
     if bound == "tensor":
         ar = d["attention_roofline"]                            # the round also reports its exp2-bound kernel
         assert ar["bound"] == "alu" and ar["peak"] > 0 and 0 < ar["frac"] < 1.5
+        # the default line carries the other two parts of the metric: verifier GB/s and images/s of whole trajectories
+        for k in ("standalone", "fused"):
+            v = d["verifier_roofline"][k]
+            assert v["bound"] == "hbm" and v["launches"] == 20 and v["achieved"] > 0 and abs(v["frac"] - v["achieved"] / v["peak"]) < 1e-9
+        tr = d["trajectory"]
+        assert tr["all_accepted"]["images_per_s"] > 0 and tr["sequential_K0"]["images_per_s"] > 0
+        assert tr["sequential_K0"]["rounds"] == 250 and tr["all_accepted"]["rounds"] < 40 and tr["all_accepted"]["rejected"] == 0
+        assert len(d["kernels"]) >= 10 and abs(sum(k["share"] for k in d["kernels"]) - 1.0) < 1e-2
     e = d["e2e"]
     assert e["value"] > 0 and e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] > 0 and e["unit"] == d["unit"]
     assert {"sm_mhz", "sm_max_mhz", "reasons"} <= set(d["clocks"])
     if "--no-cpu-baseline" not in args:
         c = d["cpu_baseline"]
         assert c["kind"] == "oracle" and c["value"] > 0 and c["cores"] >= 1 and c["sample"]
+
+
+def test_verifier_sweep_line():
+    d = _line("--workload", "verifier_sweep", "--K", "6", "--batch", "64")
+    assert [p["mode"] for p in d["points"]] == ["strict", "relaxed"]
+    assert all(p["gbs"] > 0 and p["K"] == 6 and p["B"] == 64 for p in d["points"])
