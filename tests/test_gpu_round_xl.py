@@ -10,12 +10,18 @@ from gpu_util import cu, nerr, rms_rel
 
 pytestmark = pytest.mark.gpu
 TOL = 2e-2
-# RMS-relative bound.  A bf16 rounding has relative RMS error 2^-9/sqrt(3) = 1.1e-3.  A block rounds four GEMM operands
-# (modulated LayerNorm output twice, attention output, MLP hidden) plus q/k/v and P; the branch outputs enter the fp32
-# residual stream through gates of RMS ~ 0.1 * |SiLU(c)| and are renormalised by the next LayerNorm, so the relative
-# error of the stream grows like a random walk over 28 x ~6 roundings: 1.1e-3 * sqrt(168) = 1.5e-2 if every rounding
-# came through at full weight.  The gates pass well under half of it; 1e-2 leaves that margin and is half of TOL.
-TOL_RMS = 1e-2
+# RMS-relative bounds (sqrt(mean err^2) / sqrt(mean ref^2); unlike the max-normalised measure they see an error confined
+# to small elements).  Feature: a bf16 rounding has relative RMS error 2^-9/sqrt(3) = 1.1e-3.  A block rounds four GEMM
+# operands (modulated LayerNorm output twice, attention output, MLP hidden) plus q/k/v and P; the branch outputs enter
+# the fp32 residual stream through gates of RMS ~ 0.1 |SiLU(c)| and are renormalised by the next LayerNorm, so the
+# relative error of the stream grows like a random walk over 28 x ~6 roundings: 1.1e-3 sqrt(168) = 1.5e-2 if every
+# rounding came through at full weight; the gates pass well under half of it: 1e-2.
+# Noise prediction and mean: the head is linear in the normalised feature and accumulates at fp32 level, so each
+# stream's noise carries the feature's relative error e_f; guidance eps_u + w (eps_c - eps_u) at w = 4 adds the two
+# streams' independent errors with weights w and w - 1, sqrt(16 + 9) = 5 e_f relative to a stream's norm, which the
+# guided norm does not exceed by much when the two streams are close.  5 x 3e-3 (the feature's measured error) = 1.5e-2:
+# the bound is the 2e-2 the bf16 mode is held to, not a tighter one.
+TOL_RMS_FEAT, TOL_RMS_EPS = 1e-2, 2e-2
 
 
 @pytest.fixture(scope="module")
@@ -46,7 +52,7 @@ def test_xl_512_packed_pass_sampled_against_oracle(xl):
         errs = (nerr(eps[st], eo[i]), nerr(mean[st], mo[i]), nerr(feat[st], fo[i]))
         rms = (rms_rel(eps[st], eo[i]), rms_rel(mean[st], mo[i]), rms_rel(feat[st], fo[i]))
         print("XL/2 512 state %d: max-normalised eps/mean/feat %s  RMS-relative %s" % (st, errs, rms))
-        assert max(errs) < TOL and max(rms) < TOL_RMS
+        assert max(errs) < TOL and max(rms[:2]) < TOL_RMS_EPS and rms[2] < TOL_RMS_FEAT
     pick = [37]
     # batch invariance at full size: the same state alone gives the same result
     one = model.dit_verify_pass(cu(X[pick]), cu(T[pick], torch.int32), cu(Y[pick], torch.int32), 4.0, dsched)
@@ -110,4 +116,4 @@ def test_xl_256_packed_pass_sampled_against_oracle():
         errs = (nerr(eps[st], eo[i]), nerr(mean[st], mo[i]), nerr(feat[st], fo[i]))
         rms = (rms_rel(eps[st], eo[i]), rms_rel(mean[st], mo[i]), rms_rel(feat[st], fo[i]))
         print("XL/2 256 state %d: max-normalised eps/mean/feat %s  RMS-relative %s" % (st, errs, rms))
-        assert max(errs) < TOL and max(rms) < TOL_RMS
+        assert max(errs) < TOL and max(rms[:2]) < TOL_RMS_EPS and rms[2] < TOL_RMS_FEAT
