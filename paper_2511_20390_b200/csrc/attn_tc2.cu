@@ -130,15 +130,15 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
     const uint32_t tmem_base = *tmem_slot;
     auto fail = [&]() { *abort_flag = 1; atomicOr(a.err, FREE_DEV_ERR_ATTN); };
     // warp-uniform bounded wait; false = give up
-    auto wait = [&](uint64_t* bar, uint32_t parity) -> bool {
-        return __all_sync(0xffffffffu, !*abort_flag && tc::mbar_wait(bar, parity));
-    };
+    auto wait = [&](uint64_t* bar, uint32_t parity) -> bool { return tc::wait_uniform(bar, parity, abort_flag); };
     // two barriers polled together (their poll latencies overlap)
     auto wait2 = [&](uint64_t* b0, uint32_t p0, uint64_t* b1, uint32_t p1) -> bool {
-        if (*abort_flag) return false;
         bool r0 = tc::mbar_try_wait(b0, p0), r1 = tc::mbar_try_wait(b1, p1);
-        if (!r0) r0 = tc::mbar_wait(b0, p0);
-        if (!r1) r1 = tc::mbar_wait(b1, p1);
+        if (!(r0 && r1)) {
+            if (*abort_flag) return false;
+            if (!r0) r0 = tc::mbar_wait(b0, p0);
+            if (!r1) r1 = tc::mbar_wait(b1, p1);
+        }
         return __all_sync(0xffffffffu, r0 && r1);
     };
 

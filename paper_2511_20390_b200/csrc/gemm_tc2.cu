@@ -147,7 +147,7 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
             const int a_row = m_blk * 256 + (int)rank * 128, w_row = n_blk * BN + (int)rank * half;
             const uint32_t tx = 2u * (kABytes + (uint32_t)half * BK * 2u);
             for (int kb = 0; kb < nk; ++kb) {
-                ok = __all_sync(0xffffffffu, !*abort_flag && tc::mbar_wait(&empty[s], ph ^ 1u));
+                ok = tc::wait_uniform(&empty[s], ph ^ 1u, abort_flag);
                 if (!ok) { if (lane == 0) fail(FREE_DEV_ERR_EMPTY_WAIT); break; }
                 if (tc::elect_one()) {
                     const uint32_t dst = tc::smem_u32(tiles + (size_t)s * kStageBytes);
@@ -174,13 +174,13 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
             bool ok = true;
             for (long long t = first; ok && t < total; t += step, ++tl) {
                 const uint32_t acc = tl & 1u, aph = (tl >> 1) & 1u;
-                ok = __all_sync(0xffffffffu, !*abort_flag && tc::mbar_wait(&acce[acc], aph ^ 1u));
+                ok = tc::wait_uniform(&acce[acc], aph ^ 1u, abort_flag);
                 if (!ok) { if (lane == 0) fail(FREE_DEV_ERR_ACC_EMPTY); break; }
                 tc::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * (uint32_t)BN;
                 const uint32_t idesc = (int)(t % a.num_n) == a.num_n - 1 ? idesc_last : idesc_full;
                 for (int kb = 0; kb < nk; ++kb) {
-                    ok = __all_sync(0xffffffffu, !*abort_flag && tc::mbar_wait(&full[s], ph));
+                    ok = tc::wait_uniform(&full[s], ph, abort_flag);
                     if (!ok) { if (lane == 0) fail(FREE_DEV_ERR_FULL_WAIT); break; }
                     tc::tc_fence_after();
                     if (tc::elect_one()) {
@@ -217,8 +217,7 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
         for (long long t = first; t < total; t += step, ++tl) {
             const int m_blk = (int)(t / a.num_n), n_blk = (int)(t % a.num_n);
             const uint32_t acc = tl & 1u, aph = (tl >> 1) & 1u;
-            const bool bad = *abort_flag || !tc::mbar_wait(&accf[acc], aph);
-            if (__any_sync(0xffffffffu, bad)) { if (lane == 0) fail(FREE_DEV_ERR_ACC_FULL); break; }
+            if (!tc::wait_uniform(&accf[acc], aph, abort_flag)) { if (lane == 0) fail(FREE_DEV_ERR_ACC_FULL); break; }
             tc::tc_fence_after();
             const int row0 = m_blk * 256 + (int)rank * 128 + q * 32;
             const int row = row0 + lane;

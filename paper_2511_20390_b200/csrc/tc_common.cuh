@@ -61,6 +61,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long l
     }
 }
 
+// Warp-uniform bounded wait used by the pipelines: false = give up.  A phase that is already complete costs one poll; the
+// kernel's abort flag (a shared-memory round trip of ~50 clocks) is only read before the warp settles down to spin.
+__device__ __forceinline__ bool wait_uniform(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+    bool r = mbar_try_wait(bar, parity);
+    if (!r) r = !*abort_flag && mbar_wait(bar, parity);
+    return __all_sync(0xffffffffu, r);
+}
+
 // ---- TMA ------------------------------------------------------------------------------------------
 __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int x, int y) {
     asm volatile(
