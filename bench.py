@@ -36,6 +36,7 @@ def parse():
     ap.add_argument("--chunk", type=int, default=0, help="verifier_fused: drafts per early-exit chunk (0 = off)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="default workload: skip the verifier and trajectory measurements")
+    ap.add_argument("--no-launch-overlap", action="store_true", help="launch every kernel fully serialised (no programmatic dependent launch)")
     ap.add_argument("--K", type=int, default=0, help="verifier workloads: drafts per sample (0 = 16)")
     return ap.parse_args()
 
@@ -468,6 +469,8 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     import paper_2511_20390_b200 as free
     free.lib()        # fail loudly if the CUDA library is not built
+    if args.no_launch_overlap:
+        free.lib().free_set_launch_overlap(0)
     if args.workload == "trajectory":     # whole trajectories have their own protocol (one step takes tens of seconds)
         if rank == 0:
             from bench_round import run_trajectory
@@ -541,6 +544,7 @@ def main():
             # the other two parts of the metric, measured in this process: verifier HBM GB/s and images/s
             if hasattr(wl, "trajectory_extras"):
                 out["trajectory"] = wl.trajectory_extras()
+                out["latency_b1"] = wl.latency_extras()
             out["verifier_roofline"] = verifier_extras(peaks)
         if world == 1 and not args.no_cpu_baseline:
             v, sample = wl.oracle_sample()

@@ -171,6 +171,21 @@ class RoundWorkload:
         return {"unit": "images/s", "api": "sample_trajectory", "transitions": N_SCHED, "batch": self.B, "K": K_DRAFTS,
                 "timing": "CUDA events around the blocking call (one host synchronisation per round inside)", **out}
 
+    def latency_extras(self):
+        """Batch 1 (the regime where a single step under-fills the GPU): milliseconds per sequential step (K = 0) and per
+        speculative round (K = 6, every draft accepted) of whole 250-transition trajectories, launched kernel by kernel
+        and with the rounds replayed as a CUDA graph."""
+        out = {"unit": "ms", "batch": 1, "api": "sample_trajectory"}
+        for mode, graph in (("eager", False), ("graph", True)):
+            r = time_trajectories(self.model, self.shape, 1, {"all_accepted": (K_DRAFTS, 0.0), "sequential_K0": (0, None)},
+                                  use_graph=graph, warm=False)
+            out[mode] = {"ms_per_sequential_step": 1e3 * r["sequential_K0"]["seconds"] / r["sequential_K0"]["rounds"],
+                         "ms_per_round": 1e3 * r["all_accepted"]["seconds"] / r["all_accepted"]["rounds"],
+                         "seconds_per_image_sequential": r["sequential_K0"]["seconds"],
+                         "seconds_per_image_all_accepted": r["all_accepted"]["seconds"],
+                         "graph_rounds": r["all_accepted"]["graph_rounds"] + r["sequential_K0"]["graph_rounds"]}
+        return out
+
     def oracle_sample(self):
         return oracle_dit_sample(self.shape)
 

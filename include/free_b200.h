@@ -357,6 +357,15 @@ int free_profile_begin(free_ctx* ctx);
 int free_profile_end(free_ctx* ctx, free_prof_entry* out, int max_entries, int* n_entries);
 
 /*
+ * free_set_launch_overlap -- process-wide switch for programmatic dependent launch (a CUDA stream feature; the paper has no
+ * counterpart).  When on (the default) the kernels of a pass are launched so that each may be brought onto the SMs and
+ * do its set-up while its predecessor on the stream is still finishing; it reads and writes global memory only after the
+ * predecessor has completed, so results are identical.  It shortens a step where kernels are short (small batches).
+ * Returns the previous setting.  HOST-only; takes effect for launches made afterwards.
+ */
+int free_set_launch_overlap(int on);
+
+/*
  * Device error word (safety aid; the paper has no counterpart).  free_device_error_code() maps a HOST copy of a device
  * error word to the library's return code: 0 -> FREE_OK, anything else -> FREE_ERR_DEVICE_TIMEOUT.  It is the mapping
  * sample_trajectory() applies after every round.

@@ -92,6 +92,7 @@ _SIGNATURES = {
     "free_drafter_loss_workspace_bytes": (C.c_size_t, []),
     "free_drafter_loss": (C.c_int, [C.c_int] * 4 + [C.c_int64] + [C.c_void_p] * 4 + [C.c_float] * 4 +
                           [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "free_set_launch_overlap": (C.c_int, [C.c_int]),
     "free_device_error_code": (C.c_int, [C.c_uint32]),
     "free_selftest_bounded_wait": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]),
     "free_profile_begin": (C.c_int, [C.c_void_p]),

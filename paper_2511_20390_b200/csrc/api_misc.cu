@@ -3,6 +3,11 @@
 #include <vector>
 #include <cmath>
 
+#include <atomic>
+static std::atomic<int> g_launch_overlap{1};
+bool free_launch_overlap_enabled() { return g_launch_overlap.load(std::memory_order_relaxed) != 0; }
+extern "C" int free_set_launch_overlap(int on) { return g_launch_overlap.exchange(on ? 1 : 0); }
+
 extern "C" const char* free_strerror(int code) {
     switch (code) {
         case FREE_OK: return "ok";

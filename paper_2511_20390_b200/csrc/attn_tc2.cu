@@ -129,6 +129,9 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
     tc::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     auto fail = [&]() { *abort_flag = 1; atomicOr(a.err, FREE_DEV_ERR_ATTN); };
+    // everything above touched only this CTA's shared and tensor memory: from here on q, k, v are read
+    free_grid_dep_wait();
+    free_grid_dep_launch();
     // warp-uniform bounded wait; false = give up
     auto wait = [&](uint64_t* bar, uint32_t parity) -> bool { return tc::wait_uniform(bar, parity, abort_flag); };
     // two barriers polled together (their poll latencies overlap)
@@ -506,8 +509,7 @@ int launch(int n_seq, int n_tok, int heads, int d_head, const void* qk, long lon
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { (void)cudaGetLastError(); sms = 148; }
     const bool uniform = n_tok % (2 * BQ) == 0;
     const unsigned grid = (unsigned)((uniform && n_items > sms) ? sms : n_items);
-    attention_tc2_kernel<DP><<<grid, kThreads, G::SMEM, s>>>(mQK0, mQK1, mV, mO, a);
-    return free_check_launch();
+    return free_launch(attention_tc2_kernel<DP>, dim3(grid), dim3(kThreads), (size_t)G::SMEM, s, mQK0, mQK1, mV, mO, a);
 }
 
 }  // namespace

@@ -24,6 +24,35 @@ static inline int free_check_launch() {
 
 static inline size_t free_round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// ---- programmatic dependent launch ---------------------------------------------------------------------------
+// The kernels of a pass form a chain on one stream, and at small batches the gaps between them (launch latency, the
+// set-up of barriers, tensor memory and descriptors, the tail of the last wave) are a large part of a step.  A kernel
+// launched with free_launch(overlap = true) may be brought onto the SMs while its predecessor in the stream is still
+// running: it does its set-up, then calls free_grid_dep_wait(), which returns once the predecessor has completed and its
+// writes are visible, and then lets its own successor come up early in turn (free_grid_dep_launch()).  Both calls do
+// nothing in a kernel that was launched the ordinary way.  Nothing before free_grid_dep_wait() may read or write
+// global memory that another kernel of the stream touches.
+#ifdef __CUDACC__
+__device__ __forceinline__ void free_grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void free_grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+bool free_launch_overlap_enabled();      // process-wide switch (free_set_launch_overlap), on by default
+
+template <typename... KArgs, typename... Args>
+static inline int free_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = free_launch_overlap_enabled() ? 1 : 0;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return FREE_ERR_CUDA; }
+    return FREE_OK;
+}
+#endif
+
 __device__ __forceinline__ float free_gelu_tanh(float a) {
     // 0.5 a (1 + tanh(sqrt(2/pi) (a + 0.044715 a^3)))
     const float k0 = 0.7978845608028654f, k1 = 0.044715f;

@@ -59,6 +59,7 @@ struct Workspace {
     float *x_cur, *m_a, *pack_in, *x_draft, *m_draft, *sigma2_bk, *lam_bk, *u_bk, *cx_bk, *ce_bk, *ell_bk, *d2_bk;
     void *feat0, *feat1;
     int32_t *cur_a, *nv, *n_acc, *t_step, *t_pack, *lab_pack, *t_draft, *act_draft, *active;
+    int32_t* report;           // what the host reads after a round, contiguous: error word, then active, nv, n_acc, cursor of every sample
     size_t total;
 };
 
@@ -110,6 +111,7 @@ Workspace plan(const free_ctx* c, int n, void* base) {
     w.feat1 = take(M * D * as);
     for (int32_t** p : {&w.cur_a, &w.nv, &w.n_acc, &w.t_step, &w.t_pack, &w.lab_pack, &w.t_draft, &w.act_draft, &w.active})
         *p = (int32_t*)take((size_t)n * 4 + 256);
+    w.report = (int32_t*)take((4 + 4 * (size_t)n) * 4);
     w.total = off;
     return w;
 }
@@ -381,13 +383,22 @@ __global__ void target_sample_kernel(int B, int K, int d, int N, const int32_t* 
 }
 
 // a <- a + 1 + (finalised drafts): accepted ones plus the reflected one if a rejection occurred
-__global__ void cursor_update_kernel(int B, const int32_t* active, const int32_t* nv, const int32_t* n_acc, int32_t* cur_a) {
+// Also gathers what the host needs after a round into one contiguous record (report[0] = device error word, then the
+// B-long arrays active, nv, n_acc, cursor), so that the sampling loop reads it with a single copy.
+__global__ void cursor_update_kernel(int B, const int32_t* active, const int32_t* nv, const int32_t* n_acc, int32_t* cur_a,
+                                     const uint32_t* err, int32_t* report) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= B || !active[b]) return;
-    const int v = nv[b];
-    int fin = 0;
-    if (v > 0) { const int na = n_acc[b]; fin = na < 0 ? 0 : (na + 1 < v ? na + 1 : v); }
-    cur_a[b] += 1 + fin;
+    if (b == 0) report[0] = (int32_t)*err;
+    if (b >= B) return;
+    const int act = active[b], v = nv[b], na = n_acc[b];
+    int a = cur_a[b];
+    if (act) {
+        int fin = 0;
+        if (v > 0) fin = na < 0 ? 0 : (na + 1 < v ? na + 1 : v);
+        a += 1 + fin;
+        cur_a[b] = a;
+    }
+    report[4 + b] = act; report[4 + B + b] = v; report[4 + 2 * B + b] = na; report[4 + 3 * B + b] = a;
 }
 
 // x_hat_{a+i+1} = m_hat_{a+i+1} + sigma z_D (drafting step i).  Written as verifier operand i and, unless it is
@@ -579,7 +590,7 @@ int one_round(const free_ctx* c, const Workspace& w, const RoundIO& r, cudaStrea
                                             w.x_cur, w.n_acc, w.ell_bk, w.d2_bk, nullptr, s)); }
     }
     Scope p(c, PC_CTRL, 0, s);
-    cursor_update_kernel<<<(B + 127) / 128, 128, 0, s>>>(B, w.active, w.nv, w.n_acc, w.cur_a);
+    cursor_update_kernel<<<(B + 127) / 128, 128, 0, s>>>(B, w.active, w.nv, w.n_acc, w.cur_a, w.err, w.report);
     return free_check_launch();
 }
 
@@ -637,6 +648,13 @@ int run_trajectory(free_ctx* c, int B, const float* x0, const int32_t* labels, c
     fill_i32_kernel<<<(B + 127) / 128, 128, 0, s>>>(B, 1, w.cur_a);
     FREE_TRY(free_check_launch());
     std::vector<int32_t> h_a(B, 1), h_prev(B, 1), h_nv(B), h_acc(B), h_act(B);
+    // one pinned record per round instead of five pageable copies (each of which the driver stages and waits for)
+    struct Pinned {
+        int32_t* p = nullptr;
+        ~Pinned() { if (p) cudaFreeHost(p); }
+    } rep;
+    const size_t rep_words = 4 + 4 * (size_t)B;
+    FREE_CUDA_TRY(cudaHostAlloc((void**)&rep.p, rep_words * 4, cudaHostAllocDefault));
     std::vector<float> h_ell, h_d2, h_ce(N);
     if (diag && K > 0) {
         h_ell.resize((size_t)B * K); h_d2.resize((size_t)B * K);
@@ -680,18 +698,16 @@ int run_trajectory(free_ctx* c, int B, const float* x0, const int32_t* labels, c
         } else {
             FREE_TRY(one_round(c, w, r, s));
         }
-        FREE_CUDA_TRY(cudaMemcpyAsync(h_act.data(), w.active, B * 4, cudaMemcpyDeviceToHost, s));
-        FREE_CUDA_TRY(cudaMemcpyAsync(h_nv.data(), w.nv, B * 4, cudaMemcpyDeviceToHost, s));
-        if (K > 0) FREE_CUDA_TRY(cudaMemcpyAsync(h_acc.data(), w.n_acc, B * 4, cudaMemcpyDeviceToHost, s));
-        FREE_CUDA_TRY(cudaMemcpyAsync(h_a.data(), w.cur_a, B * 4, cudaMemcpyDeviceToHost, s));
+        FREE_CUDA_TRY(cudaMemcpyAsync(rep.p, w.report, rep_words * 4, cudaMemcpyDeviceToHost, s));
         if (diag && K > 0) {
             FREE_CUDA_TRY(cudaMemcpyAsync(h_ell.data(), w.ell_bk, (size_t)B * K * 4, cudaMemcpyDeviceToHost, s));
             FREE_CUDA_TRY(cudaMemcpyAsync(h_d2.data(), w.d2_bk, (size_t)B * K * 4, cudaMemcpyDeviceToHost, s));
         }
-        uint32_t dev_err = 0;
-        FREE_CUDA_TRY(cudaMemcpyAsync(&dev_err, w.err, 4, cudaMemcpyDeviceToHost, s));
         FREE_CUDA_TRY(cudaStreamSynchronize(s));
-        FREE_TRY(free_device_error_code(dev_err));
+        FREE_TRY(free_device_error_code((uint32_t)rep.p[0]));
+        for (int b = 0; b < B; ++b) {
+            h_act[b] = rep.p[4 + b]; h_nv[b] = rep.p[4 + B + b]; h_acc[b] = rep.p[4 + 2 * B + b]; h_a[b] = rep.p[4 + 3 * B + b];
+        }
         for (int b = 0; b < B; ++b) {
             if (!h_act[b]) continue;
             if (K > 0 && h_nv[b] > 0 && h_acc[b] < 0) return h_acc[b];

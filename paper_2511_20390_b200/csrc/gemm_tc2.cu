@@ -131,6 +131,9 @@ linear_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
     tc::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     auto fail = [&](uint32_t code) { *abort_flag = 1; atomicOr(a.err, code); };
+    // everything above touched only this cluster's shared and tensor memory: from here on the operands are read
+    free_grid_dep_wait();
+    free_grid_dep_launch();
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
@@ -383,8 +386,7 @@ int launch(const CUtensorMap& mA, const CUtensorMap& mW, const CUtensorMap& mWl,
     const long long tiles = (long long)a.num_m * a.num_n;
     const long long pairs = sm_count() / 2;
     const int grid = 2 * (int)(tiles < pairs ? tiles : pairs);
-    linear_tc2_kernel<EPI, OUT_BF16, BN><<<grid, kThreads, smem, s>>>(mA, mW, mWl, mO, mV, a);
-    return free_check_launch();
+    return free_launch(linear_tc2_kernel<EPI, OUT_BF16, BN>, dim3(grid), dim3(kThreads), smem, s, mA, mW, mWl, mO, mV, a);
 }
 
 template <int BN>
@@ -454,5 +456,17 @@ int linear_bf16_pair(const LinearArgs& l, cudaStream_t s) {
     a.heads = l.heads; a.d_head = l.d_head; a.d_pad = l.d_pad; a.n_tok = l.n_tok;
     a.q = (__nv_bfloat16*)l.q; a.k = (__nv_bfloat16*)l.k; a.vt = (__nv_bfloat16*)l.vt;
     a.err = l.err;
+    // Column blocks of 256 keep the tensor core busiest, but a small M leaves most clusters idle in the last (or only) wave:
+    // 2048 rows x 1152 columns are 40 tiles on 74 clusters.  Blocks of 128 columns make twice as many tiles, each at about
+    // 0.68 of a wide tile's time (the K loop then runs at the shared-memory limit, the epilogue is half as long).  Taken
+    // when the estimated time (waves x relative tile time) is shorter; only for the epilogues whose column chunks do not
+    // care about the block width.
+    const bool narrow_ok = (l.epi == EPI_GATE_RESIDUAL || l.epi == EPI_BIAS || l.epi == EPI_BIAS_GELU) && l.N % 128 == 0;
+    if (narrow_ok) {
+        const long long pairs = sm_count() / 2, num_m = (l.M + 255) / 256;
+        const long long wide = num_m * ((l.N + 255) / 256), narrow = num_m * (l.N / 128);
+        const double t_wide = (double)((wide + pairs - 1) / pairs), t_narrow = 0.68 * (double)((narrow + pairs - 1) / pairs);
+        if (t_narrow < t_wide) return dispatch<128>(l, a, s);
+    }
     return dispatch<256>(l, a, s);
 }

@@ -205,6 +205,8 @@ template <typename T, int VPL, bool SPLIT = false>
 __global__ void __launch_bounds__(VPL >= 9 ? 384 : 256, VPL >= 9 ? 1 : 2)
 ln_modulate_kernel(int M, int D, int rows_per_seq, const float* __restrict__ x, const float* __restrict__ shift,
                    const float* __restrict__ scale, long long mod_stride, T* __restrict__ y) {
+    free_grid_dep_wait();                  // x is the previous kernel's output
+    free_grid_dep_launch();
     const int lane = threadIdx.x % 32;
     const int warps = gridDim.x * (blockDim.x / 32);
     const int gwarp = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
@@ -452,11 +454,10 @@ static int ln_launch(int M, int D, int rps, const float* x, const float* sh, con
     const unsigned need = (unsigned)((M + wpc - 1) / wpc), cap = vpl == 9 ? 148u : 148u * 2u;
     const unsigned grid = need < cap ? need : cap;
     switch (vpl) {
-        case 3: ln_modulate_kernel<T, 3><<<grid, 256, 0, s>>>(M, D, rps, x, sh, sc, ms, y); break;    // D = 384
-        case 9: ln_modulate_kernel<T, 9><<<grid, 384, 0, s>>>(M, D, rps, x, sh, sc, ms, y); break;    // D = 1152
-        default: ln_modulate_kernel<T, 0><<<grid, 256, 0, s>>>(M, D, rps, x, sh, sc, ms, y); break;
+        case 3: return free_launch(ln_modulate_kernel<T, 3>, dim3(grid), dim3(256), 0, s, M, D, rps, x, sh, sc, ms, y);    // D = 384
+        case 9: return free_launch(ln_modulate_kernel<T, 9>, dim3(grid), dim3(384), 0, s, M, D, rps, x, sh, sc, ms, y);    // D = 1152
+        default: return free_launch(ln_modulate_kernel<T, 0>, dim3(grid), dim3(256), 0, s, M, D, rps, x, sh, sc, ms, y);
     }
-    return free_check_launch();
 }
 
 int ln_modulate(int out_dtype, int M, int D, int rows_per_seq, const float* x, const float* shift, const float* scale,

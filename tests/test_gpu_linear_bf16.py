@@ -20,7 +20,10 @@ def _operands(M, N, K, seed):
 SHAPES = [(128, 32, 64), (128, 256, 64), (256, 192, 128), (300, 384, 192), (96, 64, 256), (1, 128, 64),
           (1000, 1152, 1152), (777, 3456, 384), (40000, 384, 64), (19500, 160, 128), (640, 4608, 1152), (512, 1152, 4608),
           (9000, 3456, 384), (6100, 4608, 128), (129, 192, 64), (300, 320, 128), (2049, 1152, 256),
-          (700, 448, 128), (515, 704, 192), (260, 256, 64)]        # last column block 192, 192 and none: every narrow width of the CTA-pair kernel
+          (700, 448, 128), (515, 704, 192), (260, 256, 64),        # last column block 192, 192 and none: every narrow width of the CTA-pair kernel
+          # few row blocks: the CTA-pair kernel takes column blocks of 128 (one sequence, the two sequences of a batch-1
+          # target step with the proj and fc2 shapes, a ragged last row block, two waves of narrow tiles)
+          (1024, 1152, 1152), (2048, 1152, 1152), (2048, 1152, 4608), (1900, 1152, 1152), (4096, 1152, 1152), (2049, 1152, 1152)]
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES)
@@ -33,7 +36,7 @@ def test_bias_fp32_out_is_exact_to_accumulation_order(M, N, K):
     assert nerr(got, ref) < 2e-6 * max(1.0, np.sqrt(K / 64))
 
 
-@pytest.mark.parametrize("M,N,K", [(300, 384, 192), (1000, 1152, 1152)])
+@pytest.mark.parametrize("M,N,K", [(300, 384, 192), (1000, 1152, 1152), (2048, 1152, 4608), (2048, 4608, 1152)])
 def test_epilogues(M, N, K):
     from paper_2511_20390_b200 import binding as b
     A, W, bias = _operands(M, N, K, 5)
