@@ -36,6 +36,9 @@ def parse():
     ap.add_argument("--chunk", type=int, default=0, help="verifier_fused: drafts per early-exit chunk (0 = off)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="default workload: skip the verifier and trajectory measurements")
+    ap.add_argument("--split", default="replicas", choices=["replicas", "drafts"],
+                    help="round workload on N > 1 GPUs: independent replicas (weak scaling, default) or ONE job whose packed "
+                         "pass is partitioned over the ranks with an all-gather of the noise predictions per round (strong scaling)")
     ap.add_argument("--no-launch-overlap", action="store_true", help="launch every kernel fully serialised (no programmatic dependent launch)")
     ap.add_argument("--K", type=int, default=0, help="verifier workloads: drafts per sample (0 = 16)")
     return ap.parse_args()
@@ -308,7 +311,7 @@ class DrafterLossWorkload:
         return nb * self.bytes_per_step / self.n / 1e9 / dt, f"{nb} of {self.n} samples of the same batch"
 
 
-def make_workload(name, batch, rank, chunk=0):
+def make_workload(name, batch, rank, chunk=0, split=None):
     if name == "drafter_loss":
         return DrafterLossWorkload(batch, rank)
     if name in ("verifier",):
@@ -320,7 +323,7 @@ def make_workload(name, batch, rank, chunk=0):
             from bench_round import RoundWorkload        # the full packed-verify round (DiT + verifier)
         except ImportError:
             return VerifierWorkload(batch, rank)
-        return RoundWorkload(batch, rank)
+        return RoundWorkload(batch, rank, split=split)
     if name == "ops":
         from bench_round import OpsWorkload
         return OpsWorkload(batch, rank)
@@ -482,7 +485,8 @@ def main():
         if rank == 0:
             verifier_sweep(args, peaks)
         return
-    wl = make_workload(args.workload, args.batch, rank, args.chunk)
+    split = (rank, world) if args.split == "drafts" and args.workload in ("default", "round") else None
+    wl = make_workload(args.workload, args.batch, rank, args.chunk, split)
 
     def barrier():
         if world > 1:
@@ -527,12 +531,14 @@ def main():
 
     ms, ms_e2e = max_over_ranks([ms, ms_e2e], "cuda")
     ms_step = ms / args.steps
-    value = whole_job_value(wl.units_per_step, world, ms_step)
-    e2e_value = whole_job_value(wl.units_per_step, world, ms_e2e / n_e2e)
+    # replicas: every rank processed its own batch; a partitioned job: the ranks shared one batch
+    ranks_of_work = 1 if getattr(wl, "scaling", "weak") == "strong" else world
+    value = whole_job_value(wl.units_per_step, ranks_of_work, ms_step)
+    e2e_value = whole_job_value(wl.units_per_step, ranks_of_work, ms_e2e / n_e2e)
 
     if rank == 0:
         out = {"metric": wl.metric, "value": value, "unit": wl.unit, "n_gpus": world, "steps": args.steps,
-               "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+               "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": getattr(wl, "scaling", "weak"),
                "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic", "config": wl.config,
                "clocks": clocks,
                "e2e": {"value": e2e_value, "unit": wl.unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},

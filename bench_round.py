@@ -36,13 +36,21 @@ class RoundWorkload:
     unit = "TFLOP/s"
     dtype = "bf16"
 
-    def __init__(self, batch, rank):
+    scaling = "weak"
+
+    def __init__(self, batch, rank, split=None):
+        """split = (rank, world): ONE job whose packed pass is partitioned over the ranks (the paper's deployment, Sec. 4:
+        drafts verified on parallel GPUs); every rank then holds the same weights and inputs, and the job's work does not
+        grow with the number of ranks (strong scaling).  Default: every rank runs its own batch (replicas)."""
         import torch
         import synth
         import paper_2511_20390_b200 as free
         self.torch, self.free = torch, free
         self.shape = synth.DIT_XL2_512
         self.B = batch or 16
+        self.split = split
+        if split:
+            rank, self.scaling = 0, "strong"          # identical seeds on every rank
         B, K, sh = self.B, K_DRAFTS, self.shape
         self.model = free.Model.random(sh, 1234 + rank, dtype="bf16", with_drafter=True)
         self.sched = free.DeviceSchedule(free.respaced_schedule(N_SCHED))
@@ -63,6 +71,10 @@ class RoundWorkload:
         self.flops = round_flops(sh, B, K, self.G)
         self.units_per_step = self.flops / 1e12
         self.config = round_config(B, K, self.G)
+        if split:
+            self.config["parallelism"] = (f"packed pass partitioned over {split[1]} ranks ({B * K // split[1]} of {B * K} states each), "
+                                          "target step, drafter and verifier replicated, one all-gather of the noise predictions per round")
+            self.eps_all = torch.empty((B * K, self.G, sh.C, sh.H, sh.W), dtype=torch.float32, device="cuda")
         # host staging for the end-to-end path: everything one round consumes.  From cursor a = 21 the round takes the
         # target's noise of transition 21 (row 20), the drafter's noise of transitions 22..27 (rows 21..26) and the
         # uniforms of the same six transitions
@@ -79,6 +91,11 @@ class RoundWorkload:
         self._prof = None
 
     def _round(self):
+        if self.split:
+            self.model.spec_round_split(self.x_cur, self.cursor, self.labels, self.sched, K_DRAFTS, CFG, self.noise_t, self.noise_d,
+                                        self.uniforms, self.split[0], self.split[1], eps_all=self.eps_all, x_next=self.x_next,
+                                        cursor_next=self.cursor_next, n_accept=self.n_acc)
+            return
         self.model.spec_round(self.x_cur, self.cursor, self.labels, self.sched, K_DRAFTS, CFG, self.noise_t, self.noise_d,
                               self.uniforms, x_next=self.x_next, cursor_next=self.cursor_next, n_accept=self.n_acc)
 

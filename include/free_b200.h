@@ -341,6 +341,37 @@ int free_spec_round(free_ctx* ctx, int B, const float* x_cur, const int32_t* cur
                     void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * free_spec_round_begin / free_spec_round_finish -- one round of Algorithm 1 with the packed target pass partitioned over
+ * `world` GPUs, the deployment the paper measures (Sec. 4, wall-clock protocol: the drafts of a round are verified on
+ * parallel GPUs, one draft per GPU when the speculation length equals the number of GPUs).  Every rank holds the same
+ * weights, inputs, noise and uniforms and calls both functions with the same arguments except `rank`:
+ *   begin   target step on the current states and the K drafter steps (replicated: they are the sequential part of a
+ *           round), then the packed target pass over THIS RANK'S share of the B*K packed states (state index b*K + k;
+ *           rank r owns the contiguous range given by free_split_range); their noise predictions are written into
+ *           eps_all at the states' own positions
+ *   (caller) all-gather eps_all over the ranks, in place: every rank contributes the slice it wrote.  The library makes
+ *           no collective call itself; the exchange is the caller's (NCCL all-gather into local memory).  No kernel of
+ *           the library reads another GPU's memory.
+ *   finish  guidance, means, verification and cursor update on the gathered predictions, replicated on every rank: all
+ *           ranks take the same decisions from the same bytes, so nothing has to be sent back.
+ * With world == 1 the pair is free_spec_round() in two halves (bit-identical results).  Between the two calls the round's
+ * state lives in the workspace: the same `ws` must be passed and nothing else may use it.
+ *   rank, world   0 <= rank < world; B*K must be a multiple of world (FREE_ERR_SHAPE otherwise)
+ *   eps_all       DEVICE fp32 [B*K, G, C, H, W] (layout of dit_verify_pass_raw), caller-owned
+ *   other arguments as for free_spec_round(); params->K >= 1.  Both calls are asynchronous.
+ * free_split_range: HOST-only; the states [lo, hi) that `rank` owns.
+ */
+int free_split_range(int n_states, int world, int rank, int* lo, int* hi);
+int free_spec_round_begin(free_ctx* ctx, int B, const float* x_cur, const int32_t* cursor, const int32_t* labels,
+                          const free_schedule* sched, const free_spec_params* params,
+                          const float* noise_target, const float* noise_draft, const float* uniforms,
+                          int rank, int world, float* eps_all, void* ws, size_t ws_bytes, void* stream);
+int free_spec_round_finish(free_ctx* ctx, int B, const int32_t* labels, const free_schedule* sched, const free_spec_params* params,
+                           const float* noise_target, const float* noise_draft, const float* uniforms,
+                           const float* eps_all, float* x_next, int32_t* cursor_next, int32_t* n_accept,
+                           void* ws, size_t ws_bytes, void* stream);
+
+/*
  * Per-kernel timing (measurement aid; the paper has no counterpart).  Between free_profile_begin() and
  * free_profile_end() every kernel launched by the context's passes is bracketed by CUDA events on the caller's
  * stream.  free_profile_end() waits for them and returns one entry per kernel class: launches, summed device time

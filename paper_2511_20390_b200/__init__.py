@@ -11,7 +11,7 @@ def __getattr__(name):
     # the binding loads the shared library on first use, so that `python -m paper_2511_20390_b200.build`
     # can run before the library exists
     if name in ("spec_verify", "spec_verify_fused", "spec_verify_host", "fit_lambda_profile", "drafter_loss", "Model", "DeviceSchedule", "lib", "FreeError",
-                "op_linear", "op_ln_modulate", "op_attention", "selftest_bounded_wait", "LIB_PATH"):
+                "op_linear", "op_ln_modulate", "op_attention", "selftest_bounded_wait", "split_range", "LIB_PATH"):
         from . import binding
         return getattr(binding, name)
     raise AttributeError(name)

@@ -83,6 +83,13 @@ _SIGNATURES = {
     "free_spec_round": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(ScheduleDesc),
                                   C.POINTER(SpecParams), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                   C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "free_split_range": (C.c_int, [C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]),
+    "free_spec_round_begin": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(ScheduleDesc),
+                                        C.POINTER(SpecParams), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p,
+                                        C.c_void_p, C.c_size_t, C.c_void_p]),
+    "free_spec_round_finish": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.POINTER(ScheduleDesc), C.POINTER(SpecParams),
+                                         C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                         C.c_void_p, C.c_size_t, C.c_void_p]),
     "free_uncertainty_profile": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.POINTER(ScheduleDesc),
                                            C.POINTER(SpecParams), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
@@ -277,6 +284,13 @@ _ACT = {FREE_FP32: torch.float32, FREE_BF16: torch.bfloat16}
 _MATRICES = ("t_w1", "t_w2", "ada_w", "qkv_w", "proj_w", "fc1_w", "fc2_w", "fada_w", "fc_w")
 
 
+def split_range(n_states: int, world: int, rank: int):
+    """The packed states [lo, hi) that `rank` of `world` owns (free_split_range)."""
+    lo, hi = C.c_int(0), C.c_int(0)
+    _check(lib().free_split_range(int(n_states), int(world), int(rank), C.byref(lo), C.byref(hi)), "free_split_range")
+    return lo.value, hi.value
+
+
 def selftest_bounded_wait(limit_cycles: int = 100_000):
     """Runs the pipelines' bounded wait once on a barrier nothing signals (free_selftest_bounded_wait).  Returns
     (error word, SM cycles waited, library return code the word maps to)."""
@@ -424,6 +438,51 @@ class Model:
                                      _ptr(noise_target), _ptr(noise_draft), _ptr(uniforms), _ptr(x_next), _ptr(cursor_next),
                                      _ptr(n_accept), _ptr(ws), ws.numel(), _stream()), "free_spec_round")
         return x_next, cursor_next, n_accept
+
+    def spec_round_begin(self, x_cur, cursor, labels, sched, K, cfg_scale, noise_target, noise_draft, uniforms, rank, world,
+                         eps_all=None, lam=None):
+        """First half of a round whose packed pass is partitioned over `world` ranks (free_spec_round_begin): target step,
+        drafter steps, and the packed pass over this rank's states, written into eps_all [B*K, G, C, H, W] in place.
+        Returns (eps_all, lo, hi)."""
+        B, sh = x_cur.shape[0], self.shape
+        _dev(x_cur, torch.float32); _dev(cursor, torch.int32); _dev(labels, torch.int32)
+        prm = SpecParams(int(K), float(cfg_scale), None if lam is None else _dev(lam, torch.float32).data_ptr())
+        lo, hi = split_range(B * int(K), world, rank)
+        if eps_all is None:
+            eps_all = torch.empty((B * int(K), self.guided(cfg_scale), sh.C, sh.H, sh.W), dtype=torch.float32, device=x_cur.device)
+        ws = self.workspace(B * int(K))
+        _check(lib().free_spec_round_begin(self.ctx, B, _ptr(x_cur), _ptr(cursor), _ptr(labels), C.byref(sched.desc), C.byref(prm),
+                                           _ptr(noise_target), _ptr(noise_draft), _ptr(uniforms), int(rank), int(world), _ptr(eps_all),
+                                           _ptr(ws), ws.numel(), _stream()), "free_spec_round_begin")
+        return eps_all, lo, hi
+
+    def spec_round_finish(self, eps_all, labels, sched, K, cfg_scale, noise_target, noise_draft, uniforms, like, lam=None,
+                          x_next=None, cursor_next=None, n_accept=None):
+        """Second half (free_spec_round_finish): verification and cursor update on the gathered predictions.  `like` is the
+        round's x_cur (shape and device of the outputs).  Returns (x_next, cursor_next, n_accept)."""
+        B = like.shape[0]
+        prm = SpecParams(int(K), float(cfg_scale), None if lam is None else _dev(lam, torch.float32).data_ptr())
+        x_next = torch.empty_like(like) if x_next is None else x_next
+        cursor_next = torch.empty(B, dtype=torch.int32, device=like.device) if cursor_next is None else cursor_next
+        n_accept = torch.zeros(B, dtype=torch.int32, device=like.device) if n_accept is None else n_accept
+        ws = self.workspace(B * int(K))
+        _check(lib().free_spec_round_finish(self.ctx, B, _ptr(labels), C.byref(sched.desc), C.byref(prm), _ptr(noise_target),
+                                            _ptr(noise_draft), _ptr(uniforms), _ptr(eps_all), _ptr(x_next), _ptr(cursor_next),
+                                            _ptr(n_accept), _ptr(ws), ws.numel(), _stream()), "free_spec_round_finish")
+        return x_next, cursor_next, n_accept
+
+    def spec_round_split(self, x_cur, cursor, labels, sched, K, cfg_scale, noise_target, noise_draft, uniforms, rank, world,
+                         lam=None, eps_all=None, x_next=None, cursor_next=None, n_accept=None, group=None):
+        """One round with the packed pass partitioned over the `world` ranks of a torch.distributed group: begin, an in-place
+        all-gather of the noise predictions (every rank contributes the slice it computed; NCCL on GPUs), finish.  Every
+        rank must pass identical inputs.  Returns (x_next, cursor_next, n_accept), identical on all ranks."""
+        eps_all, lo, hi = self.spec_round_begin(x_cur, cursor, labels, sched, K, cfg_scale, noise_target, noise_draft, uniforms,
+                                                rank, world, eps_all=eps_all, lam=lam)
+        if world > 1:
+            import torch.distributed as dist
+            dist.all_gather_into_tensor(eps_all, eps_all[lo:hi], group=group)
+        return self.spec_round_finish(eps_all, labels, sched, K, cfg_scale, noise_target, noise_draft, uniforms, x_cur, lam=lam,
+                                      x_next=x_next, cursor_next=cursor_next, n_accept=n_accept)
 
     @staticmethod
     def guided(cfg_scale: float) -> int:

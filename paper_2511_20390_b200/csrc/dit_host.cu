@@ -540,9 +540,11 @@ struct RoundIO {
     const float *noise_target, *noise_draft, *uniforms;
 };
 
-// One round of Algorithm 1 for every sample whose cursor has not passed N: target step, K drafter steps,
-// packed target pass, verification, cursor update.  State (w.x_cur, w.cur_a) lives in the workspace.
-int one_round(const free_ctx* c, const Workspace& w, const RoundIO& r, cudaStream_t s) {
+// One round of Algorithm 1 for every sample whose cursor has not passed N, in three parts: (front) index tables, target
+// step, K drafter steps; (pass) the packed target pass over a range of the B*K packed states; (back) verification and
+// cursor update.  State (w.x_cur, w.cur_a) lives in the workspace.  A single GPU runs the pass over all states; with the
+// packed states partitioned over several GPUs each runs front and back in full and the pass on its share.
+int round_front(const free_ctx* c, const Workspace& w, const RoundIO& r, cudaStream_t s) {
     const int B = r.B, K = r.K, N = r.sch->N, d = c->d_latent;
     const free_schedule* sch = r.sch;
     RoundArgs ra{B, K, N, r.labels, sch->sigma2, r.lambda, r.uniforms, sch->coef_x, sch->coef_eps, w.cur_a, w.nv, w.t_step,
@@ -576,22 +578,41 @@ int one_round(const free_ctx* c, const Workspace& w, const RoundIO& r, cudaStrea
               FREE_TRY(free_check_launch()); }
             void* tmp = f_prev; f_prev = f_next; f_next = tmp;
         }
-        // (3) one packed target pass over (x_a, x_hat_{a+1..a+K-1}), stopped at the head's output
-        PassIO pi{};
-        pi.x_in = w.pack_in; pi.x_stride = d; pi.t_idx = w.t_pack; pi.labels = w.lab_pack;
-        pi.head_raw = w.head_out;
-        FREE_TRY(target_pass(c, w, B * K, r.cfg, sch, pi, s));
-        // (4) guidance, the means m_{a+1..a+K} and the sequential verification with the first-rejection break in one
-        //     kernel; the finalised state replaces x_cur
+    }
+    return FREE_OK;
+}
+
+// (3) the packed target pass over states [lo, hi) of (x_a, x_hat_{a+1..a+K-1}) of every sample (state index b*K + k),
+//     stopped at the head's output; eps_all is the [B*K, G, d] tensor of all states' noise predictions
+int round_pass(const free_ctx* c, const Workspace& w, const RoundIO& r, int lo, int hi, float* eps_all, cudaStream_t s) {
+    if (r.K < 1 || hi <= lo) return FREE_OK;
+    const int d = c->d_latent, G = (r.cfg > 0.f && r.cfg != 1.f) ? 2 : 1;
+    PassIO pi{};
+    pi.x_in = w.pack_in + (size_t)lo * d; pi.x_stride = d; pi.t_idx = w.t_pack + lo; pi.labels = w.lab_pack + lo;
+    pi.head_raw = eps_all + (size_t)lo * G * d;
+    return target_pass(c, w, hi - lo, r.cfg, r.sch, pi, s);
+}
+
+// (4) guidance, the means m_{a+1..a+K} and the sequential verification with the first-rejection break in one kernel; the
+//     finalised state replaces x_cur; then the cursors move
+int round_back(const free_ctx* c, const Workspace& w, const RoundIO& r, const float* eps_all, cudaStream_t s) {
+    const int B = r.B, K = r.K, d = c->d_latent;
+    if (K > 0) {
         const int G = (r.cfg > 0.f && r.cfg != 1.f) ? 2 : 1;
-        { Scope p(c, PC_VERIFY, (double)B * ((2.0 + G) * K + 2) * d * 4, s);
-          FREE_TRY(spec_verify_fused_launch(B, K, d, G, r.cfg, w.head_out, w.pack_in, (long long)K * d,
-                                            w.m_draft, w.x_draft, w.cx_bk, w.ce_bk, w.sigma2_bk, w.lam_bk, w.u_bk, w.nv, 0,
-                                            w.x_cur, w.n_acc, w.ell_bk, w.d2_bk, nullptr, s)); }
+        Scope p(c, PC_VERIFY, (double)B * ((2.0 + G) * K + 2) * d * 4, s);
+        FREE_TRY(spec_verify_fused_launch(B, K, d, G, r.cfg, eps_all, w.pack_in, (long long)K * d,
+                                          w.m_draft, w.x_draft, w.cx_bk, w.ce_bk, w.sigma2_bk, w.lam_bk, w.u_bk, w.nv, 0,
+                                          w.x_cur, w.n_acc, w.ell_bk, w.d2_bk, nullptr, s));
     }
     Scope p(c, PC_CTRL, 0, s);
     cursor_update_kernel<<<(B + 127) / 128, 128, 0, s>>>(B, w.active, w.nv, w.n_acc, w.cur_a, w.err, w.report);
     return free_check_launch();
+}
+
+int one_round(const free_ctx* c, const Workspace& w, const RoundIO& r, cudaStream_t s) {
+    FREE_TRY(round_front(c, w, r, s));
+    FREE_TRY(round_pass(c, w, r, 0, r.B * r.K, w.head_out, s));
+    return round_back(c, w, r, w.head_out, s);
 }
 
 int check_round_args(const free_ctx* c, int B, int K, const free_schedule* sch, void* ws, size_t ws_bytes,
@@ -624,6 +645,54 @@ extern "C" int free_spec_round(free_ctx* c, int B, const float* x_cur, const int
     FREE_CUDA_TRY(cudaMemcpyAsync(x_next, w.x_cur, (size_t)B * d * 4, cudaMemcpyDeviceToDevice, s));
     FREE_CUDA_TRY(cudaMemcpyAsync(cursor_next, w.cur_a, (size_t)B * 4, cudaMemcpyDeviceToDevice, s));
     if (n_accept && K > 0) FREE_CUDA_TRY(cudaMemcpyAsync(n_accept, w.n_acc, (size_t)B * 4, cudaMemcpyDeviceToDevice, s));
+    return FREE_OK;
+}
+
+extern "C" int free_split_range(int n_states, int world, int rank, int* lo, int* hi) {
+    if (!lo || !hi) return FREE_ERR_ARG;
+    if (n_states < 0 || world < 1 || rank < 0 || rank >= world || n_states % world) return FREE_ERR_SHAPE;
+    const int per = n_states / world;
+    *lo = rank * per; *hi = *lo + per;
+    return FREE_OK;
+}
+
+extern "C" int free_spec_round_begin(free_ctx* c, int B, const float* x_cur, const int32_t* cursor, const int32_t* labels,
+                                     const free_schedule* sch, const free_spec_params* prm,
+                                     const float* noise_target, const float* noise_draft, const float* uniforms,
+                                     int rank, int world, float* eps_all, void* ws, size_t ws_bytes, void* stream) {
+    if (!x_cur || !cursor || !labels || !prm || !noise_target || !eps_all) return FREE_ERR_ARG;
+    if (prm->K < 1) return FREE_ERR_SHAPE;
+    FREE_TRY(check_round_args(c, B, prm->K, sch, ws, ws_bytes, noise_draft, uniforms));
+    if (!free_aligned16(eps_all)) return FREE_ERR_ALIGN;
+    int lo = 0, hi = 0;
+    FREE_TRY(free_split_range(B * prm->K, world, rank, &lo, &hi));
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const int d = c->d_latent;
+    const Workspace w = plan(c, B * prm->K, ws);
+    FREE_CUDA_TRY(cudaMemsetAsync(w.err, 0, 4, s));
+    FREE_CUDA_TRY(cudaMemcpyAsync(w.x_cur, x_cur, (size_t)B * d * 4, cudaMemcpyDeviceToDevice, s));
+    FREE_CUDA_TRY(cudaMemcpyAsync(w.cur_a, cursor, (size_t)B * 4, cudaMemcpyDeviceToDevice, s));
+    RoundIO r{B, prm->K, labels, sch, prm->cfg_scale, prm->lambda, noise_target, noise_draft, uniforms};
+    FREE_TRY(round_front(c, w, r, s));
+    return round_pass(c, w, r, lo, hi, eps_all, s);
+}
+
+extern "C" int free_spec_round_finish(free_ctx* c, int B, const int32_t* labels, const free_schedule* sch, const free_spec_params* prm,
+                                      const float* noise_target, const float* noise_draft, const float* uniforms,
+                                      const float* eps_all, float* x_next, int32_t* cursor_next, int32_t* n_accept,
+                                      void* ws, size_t ws_bytes, void* stream) {
+    if (!labels || !prm || !eps_all || !x_next || !cursor_next) return FREE_ERR_ARG;
+    if (prm->K < 1) return FREE_ERR_SHAPE;
+    FREE_TRY(check_round_args(c, B, prm->K, sch, ws, ws_bytes, noise_draft, uniforms));
+    if (!free_aligned16(eps_all) || !free_aligned16(x_next)) return FREE_ERR_ALIGN;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const int d = c->d_latent;
+    const Workspace w = plan(c, B * prm->K, ws);
+    RoundIO r{B, prm->K, labels, sch, prm->cfg_scale, prm->lambda, noise_target, noise_draft, uniforms};
+    FREE_TRY(round_back(c, w, r, eps_all, s));
+    FREE_CUDA_TRY(cudaMemcpyAsync(x_next, w.x_cur, (size_t)B * d * 4, cudaMemcpyDeviceToDevice, s));
+    FREE_CUDA_TRY(cudaMemcpyAsync(cursor_next, w.cur_a, (size_t)B * 4, cudaMemcpyDeviceToDevice, s));
+    if (n_accept) FREE_CUDA_TRY(cudaMemcpyAsync(n_accept, w.n_acc, (size_t)B * 4, cudaMemcpyDeviceToDevice, s));
     return FREE_OK;
 }
 

@@ -54,6 +54,12 @@ def test_bench_line(args, bound):
         assert c["kind"] == "oracle" and c["value"] > 0 and c["cores"] >= 1 and c["sample"]
 
 
+def test_partitioned_round_line_on_one_rank():
+    # --split drafts with a single rank: the two-call round with nothing to exchange; the job's work is not multiplied
+    d = _line("--batch", "1", "--steps", "2", "--split", "drafts", "--no-cpu-baseline", "--no-extras")
+    assert d["scaling"] == "strong" and "partitioned over 1 ranks" in d["config"]["parallelism"] and d["value"] > 0
+
+
 def test_verifier_sweep_line():
     d = _line("--workload", "verifier_sweep", "--K", "6", "--batch", "64")
     assert [p["mode"] for p in d["points"]] == ["strict", "relaxed"]
