@@ -456,16 +456,20 @@ int linear_bf16_pair(const LinearArgs& l, cudaStream_t s) {
     a.heads = l.heads; a.d_head = l.d_head; a.d_pad = l.d_pad; a.n_tok = l.n_tok;
     a.q = (__nv_bfloat16*)l.q; a.k = (__nv_bfloat16*)l.k; a.vt = (__nv_bfloat16*)l.vt;
     a.err = l.err;
-    // Column blocks of 256 keep the tensor core busiest, but a small M leaves most clusters idle in the last (or only) wave:
-    // 2048 rows x 1152 columns are 40 tiles on 74 clusters.  Blocks of 128 columns make twice as many tiles, each at about
-    // 0.68 of a wide tile's time (the K loop then runs at the shared-memory limit, the epilogue is half as long).  Taken
-    // when the estimated time (waves x relative tile time) is shorter; only for the epilogues whose column chunks do not
-    // care about the block width.
+    // Column blocks of 256 keep the tensor core busiest, but few row blocks leave clusters idle in the last (or only) wave:
+    // 2048 rows x 1152 columns are 40 tiles on 74 clusters.  Blocks of 128 columns make twice as many tiles.  A narrow
+    // tile's K loop runs at the shared-memory limit (0.73 of a wide tile's, measured) and its epilogue takes half as long;
+    // with the epilogue of a wide tile worth about 1024 elements of K, the relative time of a narrow tile is
+    // (0.73 K + 0.5 * 1024) / (K + 1024): 0.62 at K = 1152, 0.69 at K = 4608 (measured: 12288 x 1152 x 1152 is 8% faster
+    // narrow, 24576 x 1152 x 1152 5% slower, 12288 x 1152 x 4608 9% slower, 2048 and 4096 x 1152 x 4608 23% faster).
+    // Narrow blocks are taken when waves x relative tile time is shorter; only
+    // for the epilogues whose column chunks do not care about the block width.
     const bool narrow_ok = (l.epi == EPI_GATE_RESIDUAL || l.epi == EPI_BIAS || l.epi == EPI_BIAS_GELU) && l.N % 128 == 0;
     if (narrow_ok) {
         const long long pairs = sm_count() / 2, num_m = (l.M + 255) / 256;
         const long long wide = num_m * ((l.N + 255) / 256), narrow = num_m * (l.N / 128);
-        const double t_wide = (double)((wide + pairs - 1) / pairs), t_narrow = 0.68 * (double)((narrow + pairs - 1) / pairs);
+        const double rel = (0.73 * l.K + 0.5 * 1024.0) / ((double)l.K + 1024.0);
+        const double t_wide = (double)((wide + pairs - 1) / pairs), t_narrow = rel * (double)((narrow + pairs - 1) / pairs);
         if (t_narrow < t_wide) return dispatch<128>(l, a, s);
     }
     return dispatch<256>(l, a, s);
