@@ -86,7 +86,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap mapQK0, const __grid_co
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t* bar_q = reinterpret_cast<uint64_t*>(smem);
-    uint64_t* bar_qz = bar_q + 1;       // Q tiles fixed up (padding columns zeroed): one arrival per softmax warp
+    uint64_t* bar_qz = bar_q + 1;       // Q tiles fixed up (padding columns zeroed): the producer warp arrives after its fix-up
     uint64_t* k_full = bar_q + 2;       // [2]
     uint64_t* k_empty = bar_q + 4;      // [2]
     uint64_t* v_full = bar_q + 6;       // [2]

@@ -14,11 +14,12 @@
 //              accumulators per CTA; stage-release and accumulator-ready barriers are signalled in both CTAs.
 //              The whole warp runs the issue loop converged and one elected lane issues: measured on B200, a
 //              single-lane (divergent) loop of wait + 4 MMAs + commit takes ~660 clocks per K step, the converged
-//              loop ~508, and one MMA cannot be issued faster than every ~94 clocks whatever its size.  Only
-//              N = 256 (128 clocks of tensor work per instruction) therefore keeps the tensor core busy, so tiles are
-//              256 wide; a ragged last column block (N = 1152 = 4.5 tiles) is computed only as wide as it is (its own
-//              tensor map of half as many W rows per CTA, its own instruction shape): it then runs at the
-//              shared-memory limit, 0.73 of a full tile's time instead of all of it;
+//              loop ~508 (= the 4 x 128 clocks the instructions take to execute).  Issuing an MMA costs the thread
+//              10-20 clocks; what a K step costs besides is its wait, fence and election, so tiles are 256 wide (128
+//              clocks of tensor work per instruction) wherever there are enough row blocks; a ragged last column block
+//              (N = 1152 = 4.5 tiles) is computed only as wide as it is (its own tensor map of half as many W rows per
+//              CTA, its own instruction shape): it then runs at the shared-memory limit, 0.73 of a full tile's time
+//              instead of all of it.  With few row blocks all column blocks are 128 wide (see linear_bf16_pair);
 //   warps 2-5  epilogue (both CTAs, each on its own 128 rows): tcgen05.ld, fused bias / GELU / gate, then
 //              through swizzled shared-memory staging to a TMA store, or a TMA add-reduction for the gated
 //              residual update (the fp32 residual stream is never read by the SM).  QKV variants: HEADS scatters
