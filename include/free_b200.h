@@ -391,7 +391,8 @@ int free_profile_end(free_ctx* ctx, free_prof_entry* out, int max_entries, int* 
  * free_set_launch_overlap -- process-wide switch for programmatic dependent launch (a CUDA stream feature; the paper has no
  * counterpart).  When on (the default) the kernels of a pass are launched so that each may be brought onto the SMs and
  * do its set-up while its predecessor on the stream is still finishing; it reads and writes global memory only after the
- * predecessor has completed, so results are identical.  It shortens a step where kernels are short (small batches).
+ * predecessor has completed, so results are identical.  It shortens a step where kernels are short and is applied to
+ * launches over at most 16384 token rows (on longer kernels it measured slightly slower).
  * Returns the previous setting.  HOST-only; takes effect for launches made afterwards.
  */
 int free_set_launch_overlap(int on);

@@ -509,7 +509,7 @@ int launch(int n_seq, int n_tok, int heads, int d_head, const void* qk, long lon
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { (void)cudaGetLastError(); sms = 148; }
     const bool uniform = n_tok % (2 * BQ) == 0;
     const unsigned grid = (unsigned)((uniform && n_items > sms) ? sms : n_items);
-    return free_launch(attention_tc2_kernel<DP>, dim3(grid), dim3(kThreads), (size_t)G::SMEM, s, mQK0, mQK1, mV, mO, a);
+    return free_launch(free_overlap_for_rows((long long)rows), attention_tc2_kernel<DP>, dim3(grid), dim3(kThreads), (size_t)G::SMEM, s, mQK0, mQK1, mV, mO, a);
 }
 
 }  // namespace

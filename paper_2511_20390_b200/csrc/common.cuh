@@ -27,7 +27,7 @@ static inline size_t free_round_up(size_t v, size_t a) { return (v + a - 1) / a 
 // ---- programmatic dependent launch ---------------------------------------------------------------------------
 // The kernels of a pass form a chain on one stream, and at small batches the gaps between them (launch latency, the
 // set-up of barriers, tensor memory and descriptors, the tail of the last wave) are a large part of a step.  A kernel
-// launched with free_launch(overlap = true) may be brought onto the SMs while its predecessor in the stream is still
+// launched with free_launch(overlap = true, ...) may be brought onto the SMs while its predecessor in the stream is still
 // running: it does its set-up, then calls free_grid_dep_wait(), which returns once the predecessor has completed and its
 // writes are visible, and then lets its own successor come up early in turn (free_grid_dep_launch()).  Both calls do
 // nothing in a kernel that was launched the ordinary way.  Nothing before free_grid_dep_wait() may read or write
@@ -37,16 +37,19 @@ __device__ __forceinline__ void free_grid_dep_wait() { asm volatile("griddepcont
 __device__ __forceinline__ void free_grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 bool free_launch_overlap_enabled();      // process-wide switch (free_set_launch_overlap), on by default
+// The early launch pays where kernels are short.  On long kernels it measured 1% SLOWER (one round of 196 608 token rows:
+// 961 against 971 TFLOP/s on one pod, the GPU at its power cap either way), so it is used up to this many token rows.
+static inline bool free_overlap_for_rows(long long rows) { return free_launch_overlap_enabled() && rows <= 16384; }
 
 template <typename... KArgs, typename... Args>
-static inline int free_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+static inline int free_launch(bool overlap, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = free_launch_overlap_enabled() ? 1 : 0;
+    cfg.numAttrs = overlap ? 1 : 0;
     const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return FREE_ERR_CUDA; }
     return FREE_OK;

@@ -387,7 +387,7 @@ int launch(const CUtensorMap& mA, const CUtensorMap& mW, const CUtensorMap& mWl,
     const long long tiles = (long long)a.num_m * a.num_n;
     const long long pairs = sm_count() / 2;
     const int grid = 2 * (int)(tiles < pairs ? tiles : pairs);
-    return free_launch(linear_tc2_kernel<EPI, OUT_BF16, BN>, dim3(grid), dim3(kThreads), smem, s, mA, mW, mWl, mO, mV, a);
+    return free_launch(free_overlap_for_rows(a.M), linear_tc2_kernel<EPI, OUT_BF16, BN>, dim3(grid), dim3(kThreads), smem, s, mA, mW, mWl, mO, mV, a);
 }
 
 template <int BN>

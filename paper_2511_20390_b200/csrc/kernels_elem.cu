@@ -454,9 +454,9 @@ static int ln_launch(int M, int D, int rps, const float* x, const float* sh, con
     const unsigned need = (unsigned)((M + wpc - 1) / wpc), cap = vpl == 9 ? 148u : 148u * 2u;
     const unsigned grid = need < cap ? need : cap;
     switch (vpl) {
-        case 3: return free_launch(ln_modulate_kernel<T, 3>, dim3(grid), dim3(256), 0, s, M, D, rps, x, sh, sc, ms, y);    // D = 384
-        case 9: return free_launch(ln_modulate_kernel<T, 9>, dim3(grid), dim3(384), 0, s, M, D, rps, x, sh, sc, ms, y);    // D = 1152
-        default: return free_launch(ln_modulate_kernel<T, 0>, dim3(grid), dim3(256), 0, s, M, D, rps, x, sh, sc, ms, y);
+        case 3: return free_launch(free_overlap_for_rows(M), ln_modulate_kernel<T, 3>, dim3(grid), dim3(256), 0, s, M, D, rps, x, sh, sc, ms, y);    // D = 384
+        case 9: return free_launch(free_overlap_for_rows(M), ln_modulate_kernel<T, 9>, dim3(grid), dim3(384), 0, s, M, D, rps, x, sh, sc, ms, y);    // D = 1152
+        default: return free_launch(free_overlap_for_rows(M), ln_modulate_kernel<T, 0>, dim3(grid), dim3(256), 0, s, M, D, rps, x, sh, sc, ms, y);
     }
 }
 
