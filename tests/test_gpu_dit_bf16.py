@@ -165,3 +165,23 @@ def test_rounds_as_cuda_graphs(free):
         graph.replay()
         torch.cuda.synchronize()
         assert all(torch.equal(a, b) for a, b in zip(out, ref)) and model.device_error() == 0
+
+
+def test_launch_overlap_does_not_change_results(free):
+    """Programmatic dependent launch only moves a kernel's set-up ahead of its predecessor's end: with the switch on or off
+    a packed pass over few token rows (where it is applied) gives the same bytes, eagerly and inside a captured round."""
+    sh, w, wd, model = _model(free, synth.DIT_S2, 41, depth=3, ada_std=0.2, out_gain=2.0)
+    N = 250
+    dsched = free.DeviceSchedule(free.respaced_schedule(N))
+    x, t, y = synth.pack_states(7, 2, 6, (sh.C, sh.H, sh.W), N, sh.n_classes)         # 12 states x 2 streams x 256 tokens = 6144 rows
+    X, T, Y = cu(x.reshape(12, sh.C, sh.H, sh.W)), cu(t.reshape(-1), torch.int32), cu(y.reshape(-1), torch.int32)
+    L = free.lib()
+    try:
+        assert L.free_set_launch_overlap(1) in (0, 1)
+        on = [a.clone() for a in model.dit_verify_pass(X, T, Y, 4.0, dsched, want_eps=True, want_feat=True)]
+        assert L.free_set_launch_overlap(0) == 1
+        off = [a.clone() for a in model.dit_verify_pass(X, T, Y, 4.0, dsched, want_eps=True, want_feat=True)]
+        torch.cuda.synchronize()
+        assert model.device_error() == 0 and all(torch.equal(a, b) for a, b in zip(on, off))
+    finally:
+        L.free_set_launch_overlap(1)
