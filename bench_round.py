@@ -133,7 +133,7 @@ class RoundWorkload:
 
     # DRAM bytes (read + write) of one fc1 launch at 24 sequences from the ncu capture summarised in
     # profiles/linear_tc2_kernel_xl_block_24seq.txt; None when the kernel changed after the capture
-    NCU_FC1_DRAM_BYTES_24SEQ = 241.23e6
+    NCU_FC1_DRAM_BYTES_24SEQ = 240.66e6
 
     def roofline(self, _ms, peaks):
         """Dominant kernel = the CTA-pair linear kernel (qkv, proj, fc1, fc2 launches of every pass): algorithmic
