@@ -473,14 +473,15 @@ class Model:
 
     def spec_round_split(self, x_cur, cursor, labels, sched, K, cfg_scale, noise_target, noise_draft, uniforms, rank, world,
                          lam=None, eps_all=None, x_next=None, cursor_next=None, n_accept=None, group=None):
-        """One round with the packed pass partitioned over the `world` ranks of a torch.distributed group: begin, an in-place
+        """One round with the packed pass partitioned over the `world` ranks of a torch.distributed group: begin, an
         all-gather of the noise predictions (every rank contributes the slice it computed; NCCL on GPUs), finish.  Every
         rank must pass identical inputs.  Returns (x_next, cursor_next, n_accept), identical on all ranks."""
         eps_all, lo, hi = self.spec_round_begin(x_cur, cursor, labels, sched, K, cfg_scale, noise_target, noise_draft, uniforms,
                                                 rank, world, eps_all=eps_all, lam=lam)
         if world > 1:
             import torch.distributed as dist
-            dist.all_gather_into_tensor(eps_all, eps_all[lo:hi], group=group)
+            # the rank's own slice is sent from a copy: not every backend takes an input that aliases the output
+            dist.all_gather_into_tensor(eps_all, eps_all[lo:hi].clone(), group=group)
         return self.spec_round_finish(eps_all, labels, sched, K, cfg_scale, noise_target, noise_draft, uniforms, x_cur, lam=lam,
                                       x_next=x_next, cursor_next=cursor_next, n_accept=n_accept)
 
